@@ -1,0 +1,134 @@
+/*
+ * pp_attn.h -- C ABI of the preference-packed attention library for B200 (sm_100a).
+ *
+ * Operation (paper Sec. 3.2, "Preference packing"): one preference sample
+ * (x, y^1 .. y^K) is laid out as a single sequence [x | y^1 | ... | y^K].  The
+ * attention mask makes the result identical to running the K sequences (x, y^k)
+ * separately: prompt tokens attend causally among themselves, a response token
+ * attends to the whole prompt and causally inside its own response, and never to
+ * another response.  Several such groups may follow each other in one row (batch
+ * packing, Sec. 2.2); attention never crosses a group boundary.  The library
+ * computes that masked softmax attention, forward and backward, touching only the
+ * (query, key) tiles the mask leaves visible.
+ *
+ * Data layout (all device memory, owned by the caller, never freed or allocated here):
+ *   tokens of all rows are concatenated; T = total tokens; no padding tokens exist.
+ *   Q, O, dO, dQ : bf16 [T][Hq][D]        K, V, dK, dV : bf16 [T][Hkv][D]
+ *   LSE          : fp32 [Hq][T], natural log of sum_j exp(scale * q_i . k_j) over visible j
+ *   query head h reads KV head h / (Hq / Hkv).
+ *   Base pointers must be 16-byte aligned.  Inputs must be finite.
+ *
+ * All functions return 0 (PP_OK) or a negative pp_status; they never throw, exit or print.
+ * Work is enqueued on the caller's stream; only pp_plan_status synchronises.
+ */
+#ifndef PP_ATTN_H_
+#define PP_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* pp_stream_t; /* a cudaStream_t */
+typedef struct pp_plan pp_plan;          /* opaque host handle; device part lives in caller memory */
+
+enum pp_status {
+  PP_OK = 0,
+  PP_ERR_INVALID_ARG = -1,         /* null pointer, non-positive length, non-monotone offsets,
+                                      total_tokens mismatch, Hq % Hkv != 0 */
+  PP_ERR_UNSUPPORTED = -2,         /* head_dim not in {64, 128}; device is not sm_100 */
+  PP_ERR_WORKSPACE_TOO_SMALL = -3, /* plan workspace or scratch smaller than the size query says */
+  PP_ERR_ALIGNMENT = -4,           /* a tensor base pointer is not 16-byte aligned */
+  PP_ERR_CUDA = -5,                /* a CUDA runtime / driver call failed */
+  PP_ERR_PLAN_STATUS = -6          /* device-side validation failed or a bounded wait expired */
+};
+
+/*
+ * Problem statement, in the paper's terms (Sec. 3.1 symbols): per group g one prompt of
+ * length P_g (l_in) and n_g >= 1 responses of lengths R_{g,1..n_g} (l_resp^k).
+ * Descriptor arrays are int32 and are read during pp_build_plan only.
+ */
+typedef struct {
+  int32_t num_rows;
+  const int32_t* row_group_off;  /* [num_rows + 1]  groups of row r = [off[r], off[r+1])      */
+  const int32_t* grp_prompt_len; /* [G]             P_g >= 1                                  */
+  const int32_t* grp_resp_off;   /* [G + 1]         responses of group g = [off[g], off[g+1]) */
+  const int32_t* resp_len;       /* [N]             R >= 1                                    */
+  int32_t num_groups;            /* G = row_group_off[num_rows]                               */
+  int32_t num_responses;         /* N = grp_resp_off[G]                                       */
+  int32_t desc_on_device;        /* 0: host arrays (validated and copied by the library);
+                                    1: device arrays (validated by the plan kernel)          */
+  int32_t num_q_heads;           /* Hq                                                        */
+  int32_t num_kv_heads;          /* Hkv, divides Hq                                           */
+  int32_t head_dim;              /* D: 64 or 128                                              */
+  int32_t total_tokens;          /* T = sum of every prompt and response length (checked)     */
+} pp_problem;
+
+/* Bytes the caller must provide: plan workspace (device, 256-byte aligned), scratch for
+ * pp_attn_fwd (may be 0) and for pp_attn_bwd (fp32 dQ accumulator, Delta, scaled LSE). */
+int pp_plan_workspace_bytes(const pp_problem* problem, size_t* plan_bytes,
+                            size_t* fwd_scratch_bytes, size_t* bwd_scratch_bytes);
+
+/*
+ * Plan builder (device side, stream ordered, no host synchronisation).  Turns the segment
+ * descriptors into query/key tiles of 128 tokens aligned to segment starts, each with the
+ * key ranges it must visit -- the prompt range and the part of its own segment before it
+ * (class FULL: no masking), then its own diagonal tile (class DIAG: causal masking) --
+ * while tiles of sibling responses are never listed (class SKIP is implicit).  The same
+ * tiles, read as key tiles, carry the contiguous query range [start, vis_end) that sees
+ * them, for the backward pass.  Tiles are ordered longest-work-first for both passes.
+ * d_workspace must stay alive and untouched while the plan is used.  The plan is
+ * immutable and can be reused by any number of pp_attn_fwd / pp_attn_bwd calls whose
+ * tensors have the shapes stated in `problem`.
+ */
+int pp_build_plan(const pp_problem* problem, void* d_workspace, size_t workspace_bytes,
+                  pp_stream_t stream, pp_plan** out_plan);
+
+/* Synchronises `stream`, then reports the device status word (0 = fine) and a detail word
+ * (site of a failed validation or of an expired wait).  Returns PP_ERR_PLAN_STATUS if the
+ * status is non-zero. */
+int pp_plan_status(const pp_plan* plan, pp_stream_t stream, int32_t* status, int32_t* detail);
+
+/* Frees the host handle only. */
+int pp_destroy_plan(pp_plan* plan);
+
+/* Debug / test access: copies the tile table to host memory after synchronising `stream`.
+ * Each tile is 8 int32: {start, len, kv0_start, kv0_len, kv1_start, kv1_len, vis_end, work}.
+ * fwd_order / bwd_order receive the processing orders (tile indices).  key_end receives,
+ * per token j, the first query index that can NOT see key j.  Any pointer may be NULL.
+ * *num_tiles receives the tile count; arrays must hold pp_plan_max_tiles entries. */
+int pp_plan_max_tiles(const pp_plan* plan);
+int pp_plan_read(const pp_plan* plan, pp_stream_t stream, int32_t* num_tiles, int32_t* tiles,
+                 int32_t* fwd_order, int32_t* bwd_order, int32_t* key_end);
+
+/*
+ * Forward (Sec. 3.2): O = softmax(mask(scale * Q K^T)) V and LSE, per row and query head.
+ * q, k, v, o: bf16 device pointers; lse: fp32 device pointer.  scratch may be NULL when the
+ * size query returned 0.
+ */
+int pp_attn_fwd(const pp_plan* plan, const void* q, const void* k, const void* v,
+                float softmax_scale, void* o, float* lse, void* d_scratch, size_t scratch_bytes,
+                pp_stream_t stream);
+
+/*
+ * Backward of the same operation (training is the paper's use case, Sec. 4-5): given dO,
+ * the forward's O and LSE, writes dQ, dK, dV (bf16).  Prompt keys receive contributions from
+ * the prompt's own queries and from every response's queries; dK and dV are summed over the
+ * query heads that share a KV head.  dQ is accumulated in fp32 inside d_scratch and rounded
+ * once at the end.
+ */
+int pp_attn_bwd(const pp_plan* plan, const void* q, const void* k, const void* v, const void* o,
+                const float* lse, const void* d_o, float softmax_scale, void* d_q, void* d_k,
+                void* d_v, void* d_scratch, size_t scratch_bytes, pp_stream_t stream);
+
+/* Kernel launches enqueued by the last pp_attn_fwd / pp_attn_bwd call of this thread. */
+int pp_last_launch_count(void);
+
+const char* pp_error_string(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PP_ATTN_H_ */

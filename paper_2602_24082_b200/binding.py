@@ -1,0 +1,228 @@
+"""Thin ctypes binding of libpp_attn.so: argument marshalling only.
+
+Every step of the path (plan building, forward, backward) runs in the library's CUDA
+kernels; PyTorch only provides device memory and the current stream.  There is no CPU
+fallback: if the library is missing or no CUDA device is present, calls raise.
+
+Function names mirror the C ABI (include/pp_attn.h): pp_build_plan, pp_attn_fwd,
+pp_attn_bwd.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence, Tuple
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpp_attn.so")
+_lib: Optional[ctypes.CDLL] = None
+
+EXPORTS = ["pp_plan_workspace_bytes", "pp_build_plan", "pp_plan_status", "pp_destroy_plan",
+           "pp_plan_max_tiles", "pp_plan_read", "pp_attn_fwd", "pp_attn_bwd",
+           "pp_last_launch_count", "pp_error_string"]
+
+
+class PPError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = lib().pp_error_string(code).decode()
+        super().__init__(f"{where}: {msg} ({code})")
+
+
+class _Problem(ctypes.Structure):
+    _fields_ = [("num_rows", ctypes.c_int32),
+                ("row_group_off", ctypes.c_void_p),
+                ("grp_prompt_len", ctypes.c_void_p),
+                ("grp_resp_off", ctypes.c_void_p),
+                ("resp_len", ctypes.c_void_p),
+                ("num_groups", ctypes.c_int32),
+                ("num_responses", ctypes.c_int32),
+                ("desc_on_device", ctypes.c_int32),
+                ("num_q_heads", ctypes.c_int32),
+                ("num_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32),
+                ("total_tokens", ctypes.c_int32)]
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the CUDA library; fails loudly when it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with "
+                               "`python -m paper_2602_24082_b200.build` (there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        L.pp_error_string.restype = ctypes.c_char_p
+        L.pp_error_string.argtypes = [ctypes.c_int]
+        vp, sz = ctypes.c_void_p, ctypes.c_size_t
+        L.pp_plan_workspace_bytes.argtypes = [vp, vp, vp, vp]
+        L.pp_build_plan.argtypes = [vp, vp, sz, vp, vp]
+        L.pp_plan_status.argtypes = [vp, vp, vp, vp]
+        L.pp_destroy_plan.argtypes = [vp]
+        L.pp_plan_max_tiles.argtypes = [vp]
+        L.pp_plan_read.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+        L.pp_attn_fwd.argtypes = [vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, sz, vp]
+        L.pp_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, sz, vp]
+        _lib = L
+    return _lib
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(rc: int, where: str):
+    if rc != 0:
+        raise PPError(rc, where)
+
+
+class Plan:
+    """Owns the host handle, the device workspace and the backward scratch of one problem."""
+
+    def __init__(self, handle: int, problem: _Problem, workspace: torch.Tensor, keep, sizes):
+        self.handle = handle
+        self.problem = problem
+        self.workspace = workspace
+        self._keep = keep
+        self.plan_bytes, self.fwd_scratch_bytes, self.bwd_scratch_bytes = sizes
+        self._bwd_scratch: Optional[torch.Tensor] = None
+
+    @property
+    def total_tokens(self) -> int:
+        return self.problem.total_tokens
+
+    def bwd_scratch(self) -> torch.Tensor:
+        if self._bwd_scratch is None:
+            self._bwd_scratch = torch.empty(self.bwd_scratch_bytes, dtype=torch.uint8,
+                                            device=self.workspace.device)
+        return self._bwd_scratch
+
+    def status(self) -> Tuple[int, int]:
+        st, det = ctypes.c_int32(0), ctypes.c_int32(0)
+        lib().pp_plan_status(self.handle, _stream(), ctypes.byref(st), ctypes.byref(det))
+        return st.value, det.value
+
+    def read(self):
+        """(tiles [n,8], fwd_order [n], bwd_order [n], key_end [T]) as numpy arrays."""
+        mt = lib().pp_plan_max_tiles(self.handle)
+        tiles = np.zeros((mt, 8), dtype=np.int32)
+        fo = np.zeros(mt, dtype=np.int32)
+        bo = np.zeros(mt, dtype=np.int32)
+        ke = np.zeros(self.total_tokens, dtype=np.int32)
+        n = ctypes.c_int32(0)
+        _check(lib().pp_plan_read(self.handle, _stream(), ctypes.byref(n), tiles.ctypes.data,
+                                  fo.ctypes.data, bo.ctypes.data, ke.ctypes.data), "pp_plan_read")
+        return tiles[:n.value], fo[:n.value], bo[:n.value], ke
+
+    def __del__(self):
+        try:
+            if self.handle:
+                lib().pp_destroy_plan(self.handle)
+                self.handle = 0
+        except Exception:
+            pass
+
+
+def make_problem(desc: Sequence[np.ndarray], num_q_heads: int, num_kv_heads: int, head_dim: int,
+                 total_tokens: int, device_arrays: Optional[Sequence[torch.Tensor]] = None):
+    """Fills a pp_problem.  ``desc`` = (row_group_off, grp_prompt_len, grp_resp_off, resp_len)."""
+    arrs = [np.ascontiguousarray(a, dtype=np.int32) for a in desc]
+    p = _Problem()
+    p.num_rows = len(arrs[0]) - 1
+    p.num_groups = len(arrs[1])
+    p.num_responses = len(arrs[3])
+    if device_arrays is not None:
+        ptrs = [t.data_ptr() for t in device_arrays]
+        p.desc_on_device = 1
+    else:
+        ptrs = [a.ctypes.data for a in arrs]
+        p.desc_on_device = 0
+    p.row_group_off, p.grp_prompt_len, p.grp_resp_off, p.resp_len = ptrs
+    p.num_q_heads, p.num_kv_heads, p.head_dim = num_q_heads, num_kv_heads, head_dim
+    p.total_tokens = total_tokens
+    return p, (arrs, device_arrays)
+
+
+def pp_plan_workspace_bytes(problem: _Problem) -> Tuple[int, int, int]:
+    a, b, c = ctypes.c_size_t(0), ctypes.c_size_t(0), ctypes.c_size_t(0)
+    _check(lib().pp_plan_workspace_bytes(ctypes.byref(problem), ctypes.byref(a), ctypes.byref(b),
+                                         ctypes.byref(c)), "pp_plan_workspace_bytes")
+    return a.value, b.value, c.value
+
+
+def pp_build_plan(desc: Sequence[np.ndarray], num_q_heads: int, num_kv_heads: int, head_dim: int,
+                  total_tokens: int, device: str = "cuda:0", desc_on_device: bool = False) -> Plan:
+    if not torch.cuda.is_available():
+        raise RuntimeError("pp_build_plan needs a CUDA device (there is no CPU fallback)")
+    dev_arrays = None
+    if desc_on_device:
+        dev_arrays = [torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device) for a in desc]
+    problem, keep = make_problem(desc, num_q_heads, num_kv_heads, head_dim, total_tokens, dev_arrays)
+    sizes = pp_plan_workspace_bytes(problem)
+    ws = torch.empty(sizes[0], dtype=torch.uint8, device=device)
+    handle = ctypes.c_void_p(0)
+    with torch.cuda.device(ws.device):
+        _check(lib().pp_build_plan(ctypes.byref(problem), ws.data_ptr(), sizes[0], _stream(),
+                                   ctypes.byref(handle)), "pp_build_plan")
+    return Plan(handle.value, problem, ws, keep, sizes)
+
+
+def _chk(t: torch.Tensor, shape, dtype, name):
+    if t.dtype != dtype or tuple(t.shape) != tuple(shape) or not t.is_contiguous() or not t.is_cuda:
+        raise ValueError(f"{name}: expected contiguous CUDA {dtype} {tuple(shape)}, got "
+                         f"{t.dtype} {tuple(t.shape)} on {t.device}")
+
+
+def pp_attn_fwd(plan: Plan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor,
+                softmax_scale: float, o: Optional[torch.Tensor] = None,
+                lse: Optional[torch.Tensor] = None):
+    p = plan.problem
+    T, Hq, Hkv, D = p.total_tokens, p.num_q_heads, p.num_kv_heads, p.head_dim
+    _chk(q, (T, Hq, D), torch.bfloat16, "q")
+    _chk(k, (T, Hkv, D), torch.bfloat16, "k")
+    _chk(v, (T, Hkv, D), torch.bfloat16, "v")
+    if o is None:
+        o = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty(Hq, T, dtype=torch.float32, device=q.device)
+    _chk(o, (T, Hq, D), torch.bfloat16, "o")
+    _chk(lse, (Hq, T), torch.float32, "lse")
+    with torch.cuda.device(q.device):
+        _check(lib().pp_attn_fwd(plan.handle, q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                 float(softmax_scale), o.data_ptr(), lse.data_ptr(), None, 0,
+                                 _stream()), "pp_attn_fwd")
+    return o, lse
+
+
+def pp_attn_bwd(plan: Plan, q, k, v, o, lse, d_o, softmax_scale: float, d_q=None, d_k=None, d_v=None):
+    p = plan.problem
+    T, Hq, Hkv, D = p.total_tokens, p.num_q_heads, p.num_kv_heads, p.head_dim
+    _chk(q, (T, Hq, D), torch.bfloat16, "q")
+    _chk(k, (T, Hkv, D), torch.bfloat16, "k")
+    _chk(v, (T, Hkv, D), torch.bfloat16, "v")
+    _chk(o, (T, Hq, D), torch.bfloat16, "o")
+    _chk(d_o, (T, Hq, D), torch.bfloat16, "d_o")
+    _chk(lse, (Hq, T), torch.float32, "lse")
+    d_q = torch.empty_like(q) if d_q is None else d_q
+    d_k = torch.empty_like(k) if d_k is None else d_k
+    d_v = torch.empty_like(v) if d_v is None else d_v
+    scratch = plan.bwd_scratch()
+    with torch.cuda.device(q.device):
+        _check(lib().pp_attn_bwd(plan.handle, q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                 o.data_ptr(), lse.data_ptr(), d_o.data_ptr(), float(softmax_scale),
+                                 d_q.data_ptr(), d_k.data_ptr(), d_v.data_ptr(), scratch.data_ptr(),
+                                 scratch.numel(), _stream()), "pp_attn_bwd")
+    return d_q, d_k, d_v
+
+
+def pp_last_launch_count() -> int:
+    return int(lib().pp_last_launch_count())
+
+
+def plan_for(workload, device: str = "cuda:0", desc_on_device: bool = False) -> Plan:
+    """Convenience: plan of a :class:`workloads.Workload`."""
+    return pp_build_plan(workload.descriptors(), workload.num_q_heads, workload.num_kv_heads,
+                         workload.head_dim, workload.total_tokens, device, desc_on_device)

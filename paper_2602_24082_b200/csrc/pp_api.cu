@@ -1,0 +1,215 @@
+// C ABI of the preference-packed attention library: argument checking, plan handle,
+// workspace bookkeeping.  All device work is enqueued by the launchers in the other files.
+#include <new>
+#include <string.h>
+
+#include "pp_internal.h"
+
+namespace {
+
+thread_local int g_last_launches = 0;
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+int check_problem_shape(const pp_problem* p) {
+  if (!p) return PP_ERR_INVALID_ARG;
+  if (p->num_rows < 1 || p->num_groups < 1 || p->num_responses < 1 || p->total_tokens < 1)
+    return PP_ERR_INVALID_ARG;
+  if (p->num_groups < p->num_rows || p->num_responses < p->num_groups) return PP_ERR_INVALID_ARG;
+  if (p->num_q_heads < 1 || p->num_kv_heads < 1 || p->num_q_heads % p->num_kv_heads != 0)
+    return PP_ERR_INVALID_ARG;
+  if (p->head_dim != 64 && p->head_dim != 128) return PP_ERR_UNSUPPORTED;
+  return PP_OK;
+}
+
+// Complete validation of host-side descriptors.
+int check_host_descriptors(const pp_problem* p) {
+  if (!p->row_group_off || !p->grp_prompt_len || !p->grp_resp_off || !p->resp_len)
+    return PP_ERR_INVALID_ARG;
+  if (p->row_group_off[0] != 0 || p->row_group_off[p->num_rows] != p->num_groups)
+    return PP_ERR_INVALID_ARG;
+  for (int r = 0; r < p->num_rows; ++r)
+    if (p->row_group_off[r + 1] <= p->row_group_off[r]) return PP_ERR_INVALID_ARG;
+  if (p->grp_resp_off[0] != 0 || p->grp_resp_off[p->num_groups] != p->num_responses)
+    return PP_ERR_INVALID_ARG;
+  long long total = 0;
+  for (int g = 0; g < p->num_groups; ++g) {
+    if (p->grp_prompt_len[g] < 1) return PP_ERR_INVALID_ARG;
+    if (p->grp_resp_off[g + 1] <= p->grp_resp_off[g]) return PP_ERR_INVALID_ARG;
+    total += p->grp_prompt_len[g];
+  }
+  for (int x = 0; x < p->num_responses; ++x) {
+    if (p->resp_len[x] < 1) return PP_ERR_INVALID_ARG;
+    total += p->resp_len[x];
+  }
+  if (total != p->total_tokens) return PP_ERR_INVALID_ARG;
+  return PP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int pp_plan_workspace_bytes(const pp_problem* problem, size_t* plan_bytes,
+                            size_t* fwd_scratch_bytes, size_t* bwd_scratch_bytes) {
+  int rc = check_problem_shape(problem);
+  if (rc) return rc;
+  if (plan_bytes) *plan_bytes = pp::plan_layout(*problem).total;
+  if (fwd_scratch_bytes) *fwd_scratch_bytes = 0;
+  if (bwd_scratch_bytes) *bwd_scratch_bytes = pp::bwd_scratch_layout(*problem).total;
+  return PP_OK;
+}
+
+int pp_build_plan(const pp_problem* problem, void* d_workspace, size_t workspace_bytes,
+                  pp_stream_t stream, pp_plan** out_plan) {
+  if (!out_plan) return PP_ERR_INVALID_ARG;
+  *out_plan = nullptr;
+  int rc = check_problem_shape(problem);
+  if (rc) return rc;
+  if (!d_workspace) return PP_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(d_workspace) & 255) return PP_ERR_ALIGNMENT;
+  if (!problem->row_group_off || !problem->grp_prompt_len || !problem->grp_resp_off ||
+      !problem->resp_len)
+    return PP_ERR_INVALID_ARG;
+  pp::PlanLayout lay = pp::plan_layout(*problem);
+  if (workspace_bytes < lay.total) return PP_ERR_WORKSPACE_TOO_SMALL;
+  if (!problem->desc_on_device) {
+    rc = check_host_descriptors(problem);
+    if (rc) return rc;
+  }
+  pp_plan* plan = new (std::nothrow) pp_plan;
+  if (!plan) return PP_ERR_CUDA;
+  plan->prob = *problem;
+  plan->nseg = problem->num_groups + problem->num_responses;
+  plan->max_tiles = pp::max_tiles_of(*problem);
+  plan->ws = static_cast<char*>(d_workspace);
+  plan->lay = lay;
+  plan->fwd_scratch = 0;
+  plan->bwd_scratch = pp::bwd_scratch_layout(*problem).total;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+
+  if (!problem->desc_on_device) {
+    // stage the four arrays in the workspace; the plan kernels read them from there
+    int32_t* d = reinterpret_cast<int32_t*>(plan->ws + lay.desc);
+    const int32_t* src[4] = {problem->row_group_off, problem->grp_prompt_len,
+                             problem->grp_resp_off, problem->resp_len};
+    size_t n[4] = {size_t(problem->num_rows) + 1, size_t(problem->num_groups),
+                   size_t(problem->num_groups) + 1, size_t(problem->num_responses)};
+    const int32_t* dst[4];
+    for (int i = 0; i < 4; ++i) {
+      cudaError_t e = cudaMemcpyAsync(d, src[i], n[i] * sizeof(int32_t), cudaMemcpyHostToDevice, s);
+      if (e != cudaSuccess) {
+        delete plan;
+        return PP_ERR_CUDA;
+      }
+      dst[i] = d;
+      d += n[i];
+    }
+    plan->prob.row_group_off = dst[0];
+    plan->prob.grp_prompt_len = dst[1];
+    plan->prob.grp_resp_off = dst[2];
+    plan->prob.resp_len = dst[3];
+  }
+  if (pp::launch_plan(plan, s) != cudaSuccess) {
+    delete plan;
+    return PP_ERR_CUDA;
+  }
+  *out_plan = plan;
+  return PP_OK;
+}
+
+int pp_plan_status(const pp_plan* plan, pp_stream_t stream, int32_t* status, int32_t* detail) {
+  if (!plan) return PP_ERR_INVALID_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  int32_t h[2] = {0, 0};
+  if (cudaMemcpyAsync(h, plan->ws + plan->lay.header, sizeof h, cudaMemcpyDeviceToHost, s) !=
+          cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess)
+    return PP_ERR_CUDA;
+  if (status) *status = h[0];
+  if (detail) *detail = h[1];
+  return h[0] == 0 ? PP_OK : PP_ERR_PLAN_STATUS;
+}
+
+int pp_destroy_plan(pp_plan* plan) {
+  delete plan;
+  return PP_OK;
+}
+
+int pp_plan_max_tiles(const pp_plan* plan) { return plan ? plan->max_tiles : PP_ERR_INVALID_ARG; }
+
+int pp_plan_read(const pp_plan* plan, pp_stream_t stream, int32_t* num_tiles, int32_t* tiles,
+                 int32_t* fwd_order, int32_t* bwd_order, int32_t* key_end) {
+  if (!plan) return PP_ERR_INVALID_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  int32_t h[4] = {0, 0, 0, 0};
+  bool ok = cudaMemcpyAsync(h, plan->ws + plan->lay.header, sizeof h, cudaMemcpyDeviceToHost, s) ==
+            cudaSuccess;
+  size_t mt = size_t(plan->max_tiles);
+  if (ok && tiles)
+    ok = cudaMemcpyAsync(tiles, plan->ws + plan->lay.tiles, mt * sizeof(pp::Tile),
+                         cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  if (ok && fwd_order)
+    ok = cudaMemcpyAsync(fwd_order, plan->ws + plan->lay.fwd_order, mt * 4, cudaMemcpyDeviceToHost,
+                         s) == cudaSuccess;
+  if (ok && bwd_order)
+    ok = cudaMemcpyAsync(bwd_order, plan->ws + plan->lay.bwd_order, mt * 4, cudaMemcpyDeviceToHost,
+                         s) == cudaSuccess;
+  if (ok && key_end)
+    ok = cudaMemcpyAsync(key_end, plan->ws + plan->lay.key_end,
+                         size_t(plan->prob.total_tokens) * 4, cudaMemcpyDeviceToHost, s) ==
+         cudaSuccess;
+  if (!ok || cudaStreamSynchronize(s) != cudaSuccess) return PP_ERR_CUDA;
+  if (num_tiles) *num_tiles = h[2];
+  return h[0] == 0 ? PP_OK : PP_ERR_PLAN_STATUS;
+}
+
+int pp_attn_fwd(const pp_plan* plan, const void* q, const void* k, const void* v,
+                float softmax_scale, void* o, float* lse, void* d_scratch, size_t scratch_bytes,
+                pp_stream_t stream) {
+  (void)d_scratch;
+  (void)scratch_bytes;
+  g_last_launches = 0;
+  if (!plan || !q || !k || !v || !o || !lse) return PP_ERR_INVALID_ARG;
+  if (!(softmax_scale > 0.f) || softmax_scale > 1e30f) return PP_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse))
+    return PP_ERR_ALIGNMENT;
+  cudaError_t e = pp::launch_fwd(plan, q, k, v, softmax_scale, o, lse,
+                                 reinterpret_cast<cudaStream_t>(stream), &g_last_launches);
+  return e == cudaSuccess ? PP_OK : (e == cudaErrorNotSupported ? PP_ERR_UNSUPPORTED : PP_ERR_CUDA);
+}
+
+int pp_attn_bwd(const pp_plan* plan, const void* q, const void* k, const void* v, const void* o,
+                const float* lse, const void* d_o, float softmax_scale, void* d_q, void* d_k,
+                void* d_v, void* d_scratch, size_t scratch_bytes, pp_stream_t stream) {
+  g_last_launches = 0;
+  if (!plan || !q || !k || !v || !o || !lse || !d_o || !d_q || !d_k || !d_v || !d_scratch)
+    return PP_ERR_INVALID_ARG;
+  if (!(softmax_scale > 0.f) || softmax_scale > 1e30f) return PP_ERR_INVALID_ARG;
+  if (scratch_bytes < plan->bwd_scratch) return PP_ERR_WORKSPACE_TOO_SMALL;
+  const void* ptrs[] = {q, k, v, o, lse, d_o, d_q, d_k, d_v};
+  for (const void* p : ptrs)
+    if (!aligned16(p)) return PP_ERR_ALIGNMENT;
+  if (reinterpret_cast<uintptr_t>(d_scratch) & 255) return PP_ERR_ALIGNMENT;
+  cudaError_t e = pp::launch_bwd(plan, q, k, v, o, lse, d_o, softmax_scale, d_q, d_k, d_v,
+                                 d_scratch, reinterpret_cast<cudaStream_t>(stream),
+                                 &g_last_launches);
+  return e == cudaSuccess ? PP_OK : (e == cudaErrorNotSupported ? PP_ERR_UNSUPPORTED : PP_ERR_CUDA);
+}
+
+int pp_last_launch_count(void) { return g_last_launches; }
+
+const char* pp_error_string(int code) {
+  switch (code) {
+    case PP_OK: return "ok";
+    case PP_ERR_INVALID_ARG: return "invalid argument";
+    case PP_ERR_UNSUPPORTED: return "unsupported head_dim or device";
+    case PP_ERR_WORKSPACE_TOO_SMALL: return "workspace or scratch too small";
+    case PP_ERR_ALIGNMENT: return "pointer not sufficiently aligned";
+    case PP_ERR_CUDA: return "CUDA call failed";
+    case PP_ERR_PLAN_STATUS: return "device-side validation failed or a bounded wait expired";
+    default: return "unknown error";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,111 @@
+// Internal definitions shared by the plan builder, the kernels and the C ABI.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/pp_attn.h"
+
+namespace pp {
+
+constexpr int kTile = 128;  // query-tile and key-tile length in tokens
+
+// One tile of a segment (prompt or response).  Read as a query tile it lists the keys it
+// sees; read as a key tile it lists the queries that see it.
+struct Tile {
+  int32_t start;      // first token
+  int32_t len;        // 1..128 tokens
+  int32_t kv0_start;  // FULL range 0: prompt keys visible to every row of the tile
+  int32_t kv0_len;    //   (for a prompt tile: the prompt keys before the tile)
+  int32_t kv1_start;  // FULL range 1: own-response keys before the tile (0 for prompt tiles)
+  int32_t kv1_len;
+  int32_t vis_end;    // queries [start, vis_end) see this tile's keys (causally inside the tile)
+  int32_t work;       // forward work estimate in key tiles (backward: derived)
+};
+static_assert(sizeof(Tile) == 32, "tile record is 32 bytes");
+
+// Status word values written by device code.
+enum : int32_t {
+  kStatusOk = 0,
+  kStatusBadDescriptor = 1,  // detail = index of the offending group / response
+  kStatusTokenMismatch = 2,  // detail = token count found
+  kStatusWaitExpired = 3,    // detail = site id
+};
+
+// Device part of a plan: offsets (bytes) into the caller's workspace.
+struct PlanLayout {
+  size_t header;     // int32[8]: status, detail, num_tiles, num_segments, ...
+  size_t desc;       // device copy of the descriptor arrays (when given on host)
+  size_t seg_start;  // int32[nseg + 1]
+  size_t seg_tile0;  // int32[nseg + 1]  first tile of each segment
+  size_t tiles;      // Tile[max_tiles]
+  size_t fwd_order;  // int32[max_tiles]
+  size_t bwd_order;  // int32[max_tiles]
+  size_t key_end;    // int32[T]
+  size_t total;
+};
+
+}  // namespace pp
+
+struct pp_plan {
+  pp_problem prob;  // descriptor pointers are rewritten to the device copies
+  int nseg;
+  int max_tiles;
+  char* ws;
+  pp::PlanLayout lay;
+  // scratch sizes
+  size_t fwd_scratch, bwd_scratch;
+};
+
+namespace pp {
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+inline int max_tiles_of(const pp_problem& p) {
+  // sum over segments of ceil(len / 128) <= T / 128 + number of segments
+  return p.total_tokens / kTile + p.num_groups + p.num_responses;
+}
+
+inline PlanLayout plan_layout(const pp_problem& p) {
+  PlanLayout l{};
+  int nseg = p.num_groups + p.num_responses;
+  int mt = max_tiles_of(p);
+  size_t off = 0;
+  l.header = off;    off = align_up(off + 64, 256);
+  l.desc = off;
+  off = align_up(off + sizeof(int32_t) * (size_t(p.num_rows) + 1 + p.num_groups +
+                                           (p.num_groups + 1) + p.num_responses), 256);
+  l.seg_start = off; off = align_up(off + sizeof(int32_t) * (nseg + 1), 256);
+  l.seg_tile0 = off; off = align_up(off + sizeof(int32_t) * (nseg + 1), 256);
+  l.tiles = off;     off = align_up(off + sizeof(Tile) * size_t(mt), 256);
+  l.fwd_order = off; off = align_up(off + sizeof(int32_t) * size_t(mt), 256);
+  l.bwd_order = off; off = align_up(off + sizeof(int32_t) * size_t(mt), 256);
+  l.key_end = off;   off = align_up(off + sizeof(int32_t) * size_t(p.total_tokens), 256);
+  l.total = off;
+  return l;
+}
+
+// Backward scratch: fp32 dQ accumulator [T][Hq][D], Delta [Hq][T], LSE*log2(e) [Hq][T]
+struct BwdScratch {
+  size_t dq_acc, delta, lse2, total;
+};
+inline BwdScratch bwd_scratch_layout(const pp_problem& p) {
+  BwdScratch s{};
+  size_t T = p.total_tokens, Hq = p.num_q_heads, D = p.head_dim;
+  size_t off = 0;
+  s.dq_acc = off; off = align_up(off + 4 * T * Hq * D, 256);
+  s.delta = off;  off = align_up(off + 4 * T * Hq, 256);
+  s.lse2 = off;   off = align_up(off + 4 * T * Hq, 256);
+  s.total = off;
+  return s;
+}
+
+// launchers (defined in the .cu files); all return a cudaError_t
+cudaError_t launch_plan(const pp_plan* plan, cudaStream_t stream);
+cudaError_t launch_fwd(const pp_plan* plan, const void* q, const void* k, const void* v, float scale,
+                       void* o, float* lse, cudaStream_t stream, int* launches);
+cudaError_t launch_bwd(const pp_plan* plan, const void* q, const void* k, const void* v,
+                       const void* o, const float* lse, const void* d_o, float scale, void* dq,
+                       void* dk, void* dv, void* scratch, cudaStream_t stream, int* launches);
+
+}  // namespace pp

@@ -1,0 +1,232 @@
+// Device-side plan builder: segment descriptors -> tiles, visible key/query ranges, orders.
+//
+// The packing mask (paper Sec. 3.2) has a simple structure once tokens are grouped by
+// segment: a key j is seen by the contiguous queries [j, end_j) where end_j is the end of
+// j's group for a prompt key and the end of j's own response otherwise; a query sees at
+// most two contiguous key ranges (its group's prompt, and its own segment up to itself).
+// Tiles are cut per segment (aligned to the segment start), so a tile never straddles two
+// segments and only its own diagonal block needs element-wise causal masking.
+#include "pp_internal.h"
+
+namespace pp {
+namespace {
+
+struct PlanPtrs {
+  int32_t* header;
+  const int32_t* row_group_off;
+  const int32_t* grp_prompt_len;
+  const int32_t* grp_resp_off;
+  const int32_t* resp_len;
+  int32_t* seg_start;
+  int32_t* seg_tile0;
+  Tile* tiles;
+  int32_t* fwd_order;
+  int32_t* bwd_order;
+  int32_t* key_end;
+  int num_rows, G, N, T, nseg, max_tiles;
+};
+
+__device__ __forceinline__ void set_status(int32_t* header, int32_t status, int32_t detail) {
+  if (atomicCAS(&header[0], kStatusOk, status) == kStatusOk) header[1] = detail;
+}
+
+// Segment order: group 0 prompt, group 0 responses, group 1 prompt, ...  so the prompt of
+// group g is segment g + resp_off[g] and response x (global index) of group g is g + 1 + x.
+
+// One block.  Validates, writes segment lengths, scans them into seg_start / seg_tile0.
+__global__ void __launch_bounds__(1024) plan_scan_kernel(PlanPtrs p) {
+  __shared__ int32_t s_tok[1024];
+  __shared__ int32_t s_til[1024];
+  __shared__ int32_t s_carry[2];
+  const int tid = threadIdx.x;
+
+  if (tid == 0) {
+    p.header[0] = kStatusOk;
+    p.header[1] = 0;
+    p.header[2] = 0;
+    p.header[3] = p.nseg;
+    if (p.row_group_off[0] != 0 || p.row_group_off[p.num_rows] != p.G)
+      set_status(p.header, kStatusBadDescriptor, -1);
+    if (p.grp_resp_off[0] != 0 || p.grp_resp_off[p.G] != p.N)
+      set_status(p.header, kStatusBadDescriptor, -2);
+    s_carry[0] = 0;
+    s_carry[1] = 0;
+  }
+  __syncthreads();
+  for (int r = tid; r < p.num_rows; r += blockDim.x)
+    if (p.row_group_off[r + 1] < p.row_group_off[r]) set_status(p.header, kStatusBadDescriptor, r);
+  // segment lengths (stored in seg_start, scanned in place below)
+  for (int g = tid; g < p.G; g += blockDim.x) {
+    int lo = p.grp_resp_off[g], hi = p.grp_resp_off[g + 1];
+    bool ok = p.grp_prompt_len[g] >= 1 && hi > lo && lo >= 0 && hi <= p.N;
+    if (!ok) {
+      set_status(p.header, kStatusBadDescriptor, g);
+      continue;
+    }
+    p.seg_start[g + lo] = p.grp_prompt_len[g];
+    for (int x = lo; x < hi; ++x) {
+      int len = p.resp_len[x];
+      if (len < 1) set_status(p.header, kStatusBadDescriptor, p.G + x);
+      p.seg_start[g + 1 + x] = len;
+    }
+  }
+  __syncthreads();
+  if (p.header[0] != kStatusOk) return;
+
+  // chunked exclusive scan of lengths and tile counts
+  for (int base = 0; base < p.nseg; base += blockDim.x) {
+    int s = base + tid;
+    int len = s < p.nseg ? p.seg_start[s] : 0;
+    // guard against overflow from absurd lengths
+    if (len > p.T) len = p.T + 1;
+    int til = (len + kTile - 1) / kTile;
+    s_tok[tid] = len;
+    s_til[tid] = til;
+    __syncthreads();
+    for (int d = 1; d < (int)blockDim.x; d <<= 1) {
+      int a = tid >= d ? s_tok[tid - d] : 0;
+      int b = tid >= d ? s_til[tid - d] : 0;
+      __syncthreads();
+      // saturate so a corrupted descriptor cannot wrap around
+      s_tok[tid] = min(s_tok[tid] + a, 0x3fffffff);
+      s_til[tid] += b;
+      __syncthreads();
+    }
+    if (s < p.nseg) {
+      p.seg_start[s] = s_carry[0] + s_tok[tid] - len;
+      p.seg_tile0[s] = s_carry[1] + s_til[tid] - til;
+    }
+    __syncthreads();
+    if (tid == blockDim.x - 1) {
+      s_carry[0] = min(s_carry[0] + s_tok[tid], 0x3fffffff);
+      s_carry[1] += s_til[tid];
+    }
+    __syncthreads();
+  }
+  if (tid == 0) {
+    p.seg_start[p.nseg] = s_carry[0];
+    p.seg_tile0[p.nseg] = s_carry[1];
+    if (s_carry[0] != p.T) {
+      set_status(p.header, kStatusTokenMismatch, s_carry[0]);
+    } else {
+      p.header[2] = s_carry[1];  // number of tiles
+    }
+  }
+}
+
+// largest s in [0, n) with a[s] <= x  (a is non-decreasing, a[0] <= x)
+__device__ __forceinline__ int upper_segment(const int32_t* a, int n, int x) {
+  int lo = 0, hi = n;
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (a[mid] <= x) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+// group of segment s: the largest g with g + resp_off[g] <= s
+__device__ __forceinline__ int group_of_segment(const PlanPtrs& p, int s) {
+  int lo = 0, hi = p.G;
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (mid + p.grp_resp_off[mid] <= s) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+__global__ void plan_tiles_kernel(PlanPtrs p) {
+  if (p.header[0] != kStatusOk) return;
+  const int ntiles = p.header[2];
+  int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= ntiles) return;
+  int s = upper_segment(p.seg_tile0, p.nseg, t);
+  // segments with zero tiles cannot exist (len >= 1), so seg_tile0 is strictly increasing
+  int g = group_of_segment(p, s);
+  int sp = g + p.grp_resp_off[g];             // the group's prompt segment
+  int gs = p.seg_start[sp];
+  int P = p.grp_prompt_len[g];
+  int gend = p.seg_start[(g + 1) + p.grp_resp_off[g + 1]];  // next group's prompt (or T)
+  int ss = p.seg_start[s], se = p.seg_start[s + 1];
+  int start = ss + (t - p.seg_tile0[s]) * kTile;
+  Tile tl;
+  tl.start = start;
+  tl.len = min(kTile, se - start);
+  if (s == sp) {
+    tl.kv0_start = gs;  tl.kv0_len = start - gs;
+    tl.kv1_start = start; tl.kv1_len = 0;
+    tl.vis_end = gend;
+  } else {
+    tl.kv0_start = gs;  tl.kv0_len = P;
+    tl.kv1_start = ss;  tl.kv1_len = start - ss;
+    tl.vis_end = se;
+  }
+  tl.work = (tl.kv0_len + kTile - 1) / kTile + (tl.kv1_len + kTile - 1) / kTile + 1;
+  p.tiles[t] = tl;
+}
+
+__global__ void plan_key_end_kernel(PlanPtrs p) {
+  if (p.header[0] != kStatusOk) return;
+  int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= p.T) return;
+  int s = upper_segment(p.seg_start, p.nseg, j);
+  int g = group_of_segment(p, s);
+  bool prompt = (s == g + p.grp_resp_off[g]);
+  p.key_end[j] = prompt ? p.seg_start[(g + 1) + p.grp_resp_off[g + 1]] : p.seg_start[s + 1];
+}
+
+__device__ __forceinline__ int bwd_work(const Tile& t) {
+  return 1 + (t.vis_end - (t.start + t.len) + kTile - 1) / kTile;
+}
+
+// Longest-work-first orders by rank counting (tile counts are small: T/128 + segments).
+__global__ void plan_order_kernel(PlanPtrs p) {
+  if (p.header[0] != kStatusOk) return;
+  const int n = p.header[2];
+  int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= n) return;
+  Tile me = p.tiles[t];
+  int wf = me.work, wb = bwd_work(me);
+  int rf = 0, rb = 0;
+  for (int u = 0; u < n; ++u) {
+    Tile o = p.tiles[u];
+    int of = o.work, ob = bwd_work(o);
+    rf += (of > wf) || (of == wf && u < t);
+    rb += (ob > wb) || (ob == wb && u < t);
+  }
+  p.fwd_order[rf] = t;
+  p.bwd_order[rb] = t;
+}
+
+}  // namespace
+
+cudaError_t launch_plan(const pp_plan* plan, cudaStream_t stream) {
+  PlanPtrs p;
+  char* ws = plan->ws;
+  const PlanLayout& l = plan->lay;
+  p.header = reinterpret_cast<int32_t*>(ws + l.header);
+  p.row_group_off = plan->prob.row_group_off;
+  p.grp_prompt_len = plan->prob.grp_prompt_len;
+  p.grp_resp_off = plan->prob.grp_resp_off;
+  p.resp_len = plan->prob.resp_len;
+  p.seg_start = reinterpret_cast<int32_t*>(ws + l.seg_start);
+  p.seg_tile0 = reinterpret_cast<int32_t*>(ws + l.seg_tile0);
+  p.tiles = reinterpret_cast<Tile*>(ws + l.tiles);
+  p.fwd_order = reinterpret_cast<int32_t*>(ws + l.fwd_order);
+  p.bwd_order = reinterpret_cast<int32_t*>(ws + l.bwd_order);
+  p.key_end = reinterpret_cast<int32_t*>(ws + l.key_end);
+  p.num_rows = plan->prob.num_rows;
+  p.G = plan->prob.num_groups;
+  p.N = plan->prob.num_responses;
+  p.T = plan->prob.total_tokens;
+  p.nseg = plan->nseg;
+  p.max_tiles = plan->max_tiles;
+
+  plan_scan_kernel<<<1, 1024, 0, stream>>>(p);
+  int mt = plan->max_tiles;
+  plan_tiles_kernel<<<(mt + 255) / 256, 256, 0, stream>>>(p);
+  plan_key_end_kernel<<<(p.T + 255) / 256, 256, 0, stream>>>(p);
+  plan_order_kernel<<<(mt + 127) / 128, 128, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace pp

@@ -1,0 +1,129 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU fp64 oracle, element by
+element on the same seeded inputs.
+
+Tolerances (for unit-normal bf16 inputs): max-abs 2e-2 on O, 5e-3 on LSE, relative L2 2e-2
+on dQ / dK / dV -- also checked per segment kind (prompt tokens only, response tokens only) so
+that an error confined to short segments cannot hide inside a global norm.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2602_24082_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+TOL_O, TOL_LSE, TOL_GRAD = 2e-2, 5e-3, 2e-2
+
+
+def _run_gpu(w, tens, desc_on_device=False):
+    from paper_2602_24082_b200 import binding as B
+    q, k, v, do = (x.cuda() for x in tens)
+    plan = B.plan_for(w, desc_on_device=desc_on_device)
+    o, lse = B.pp_attn_fwd(plan, q, k, v, w.softmax_scale)
+    dq, dk, dv = B.pp_attn_bwd(plan, q, k, v, o, lse, do, w.softmax_scale)
+    torch.cuda.synchronize()
+    assert plan.status() == (0, 0)
+    return tuple(x.float().cpu().numpy().astype(np.float64) for x in (o, lse, dq, dk, dv))
+
+
+def _rel_l2(a, b):
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-30))
+
+
+def check_against_oracle(w, tens, gpu):
+    import oracle
+    O, LSE, dQ, dK, dV = oracle.attn_fwd_bwd(w.descriptors(), *tens, w.softmax_scale)
+    o, lse, dq, dk, dv = gpu
+    assert np.isfinite(o).all() and np.isfinite(lse).all()
+    assert np.abs(o - O).max() <= TOL_O, f"O max-abs {np.abs(o - O).max()}"
+    assert np.abs(lse - LSE).max() <= TOL_LSE, f"LSE max-abs {np.abs(lse - LSE).max()}"
+    prompt = np.zeros(w.total_tokens, dtype=bool)
+    for (s, l, _, _, seg) in w.segments():
+        if seg == 0:
+            prompt[s:s + l] = True
+    for name, g, ref in (("dQ", dq, dQ), ("dK", dk, dK), ("dV", dv, dV)):
+        assert np.isfinite(g).all(), name
+        assert _rel_l2(g, ref) <= TOL_GRAD, f"{name} rel-L2 {_rel_l2(g, ref)}"
+        assert _rel_l2(g[prompt], ref[prompt]) <= TOL_GRAD, f"{name} prompt rel-L2"
+        assert _rel_l2(g[~prompt], ref[~prompt]) <= TOL_GRAD, f"{name} response rel-L2"
+
+
+def test_config0_full():
+    w = W.config0()
+    tens = w.tensors()
+    check_against_oracle(w, tens, _run_gpu(w, tens))
+
+
+RAGGED = [
+    # name, rows, Hq, Hkv, D   -- lengths around the tile size, primes, length-1 segments
+    ("d64-ragged", [[(130, (1, 127, 129))]], 2, 1, 64),
+    ("d128-ragged", [[(257, (5, 128, 31))], [(1, (1, 300))]], 4, 2, 128),
+    ("d128-groups", [[(97, (64, 200)), (128, (128, 128)), (3, (2, 1))]], 2, 2, 128),
+    ("d64-gqa4", [[(300, (140, 10, 77, 129))]], 4, 1, 64),
+    ("d128-single-response", [[(200, (333,))]], 2, 1, 128),
+]
+
+
+@pytest.mark.parametrize("name,rows,hq,hkv,d", RAGGED, ids=[r[0] for r in RAGGED])
+@pytest.mark.parametrize("desc_on_device", [False, True], ids=["hostdesc", "devdesc"])
+def test_ragged_shapes(name, rows, hq, hkv, d, desc_on_device):
+    w = W.Workload(name, rows, hq, hkv, d, seed=100 + len(name))
+    tens = w.tensors()
+    check_against_oracle(w, tens, _run_gpu(w, tens, desc_on_device))
+
+
+def _subset_parity(w, row_ids, kv_heads):
+    """Run the GPU on the whole workload, compare an independent sub-problem with the oracle."""
+    tens = w.tensors()
+    gpu = _run_gpu(w, tens)
+    sub, stens, tok, qh = W.slice_heads(w, tens, row_ids, kv_heads)
+    tok, qh = tok.numpy(), qh.numpy()
+    kh = np.asarray(kv_heads)
+    o, lse, dq, dk, dv = gpu
+    cut = (o[tok][:, qh], lse[qh][:, tok], dq[tok][:, qh], dk[tok][:, kh], dv[tok][:, kh])
+    check_against_oracle(sub, stens, cut)
+
+
+def test_config1_subset():
+    w = W.config1()
+    lens = w.row_lengths()
+    _subset_parity(w, [int(np.argmin(lens))], [3])
+
+
+def test_config1_full_rows_two_heads():
+    w = W.config1()
+    _subset_parity(w, [0, 5], [0, 7])
+
+
+def test_deterministic_forward_and_dkdv():
+    """Forward, dK and dV have a fixed summation order: two runs agree bit for bit.  dQ is
+    summed with floating-point reductions whose order may vary: compared within tolerance."""
+    w = W.Workload("det", [[(300, (140, 77))], [(64, (200, 1))]], 4, 2, 128, seed=7)
+    tens = w.tensors()
+    a = _run_gpu(w, tens)
+    b = _run_gpu(w, tens)
+    for i in (0, 1, 3, 4):
+        assert np.array_equal(a[i], b[i])
+    assert _rel_l2(a[2], b[2]) < 1e-3
+
+
+def test_outputs_outside_tiles_untouched():
+    """Guard bands: the kernels write only the rows they own."""
+    from paper_2602_24082_b200 import binding as B
+    w = W.Workload("guard", [[(70, (33, 5))]], 2, 1, 64, seed=9)
+    q, k, v, do = (x.cuda() for x in w.tensors())
+    T, Hq, Hkv, D = w.total_tokens, 2, 1, 64
+    pad = 64
+    bufs = {}
+    for name, shape in (("o", (T + 2 * pad, Hq, D)), ("dq", (T + 2 * pad, Hq, D)),
+                        ("dk", (T + 2 * pad, Hkv, D)), ("dv", (T + 2 * pad, Hkv, D))):
+        bufs[name] = torch.full(shape, 7.0, dtype=torch.bfloat16, device="cuda")
+    plan = B.plan_for(w)
+    o = bufs["o"][pad:pad + T]
+    o2, lse = B.pp_attn_fwd(plan, q, k, v, w.softmax_scale, o=o)
+    B.pp_attn_bwd(plan, q, k, v, o, lse, do, w.softmax_scale, d_q=bufs["dq"][pad:pad + T],
+                  d_k=bufs["dk"][pad:pad + T], d_v=bufs["dv"][pad:pad + T])
+    torch.cuda.synchronize()
+    for name, b in bufs.items():
+        assert (b[:pad] == 7.0).all() and (b[pad + T:] == 7.0).all(), name
