@@ -1,0 +1,419 @@
+"""Benchmark of preference-packed attention (plan + forward + backward) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config NAME]
+
+A step is one pass of the whole hot path over one synthetic batch: build the plan on the
+device from the segment descriptors, forward (O, LSE), backward (Delta preprocess, main
+kernel, dQ finalize).  The headline metric is useful TFLOP/s: 14 * Hq * D FLOPs per visible
+(query, key) pair (2 GEMMs forward, 5 backward), masked pairs inside executed tiles not
+counted.  Prints ONE JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "packed_attn_fwd_bwd_useful_tflops"
+UNIT = "TFLOP/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_BF16_TFLOPS = 1590.0
+
+# Paper figures (end-to-end training ratios on unnamed hardware): context only.
+PAPER_CONTEXT = {
+    "training_time_reduction_at_least": 0.37,
+    "speedup_with_batch_sorting": 3.22,
+    "hardware": "a single GPU (model not stated) / multi-node FSDP (GPUs not stated)",
+}
+
+
+def get_workload(name: str, rank: int = 0):
+    from paper_2602_24082_b200 import workloads as W
+    if name == "config0":
+        return W.config0()
+    if name == "config1":
+        return W.config1(seed=1 + rank)
+    if name == "config2":
+        return W.config2(seed=2 + 10 * rank)
+    if name == "config3":
+        return W.config3(seed=3 + 10 * rank)
+    if name.startswith("config4"):
+        point = int(name.split(":")[1]) if ":" in name else 0
+        return W.config4(point)
+    raise SystemExit(f"unknown config {name}")
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return float(d["bf16_tflops"]), float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "measured"
+    return FALLBACK_BF16_TFLOPS, 1400.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.005):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._halt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._halt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._halt.set()
+        self.join(timeout=2)
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def oracle_sample(w, tens, target_pairs: float = 2.0e8):
+    """A bounded, independent sub-problem of the workload for the CPU oracle: whole rows
+    (shortest first) of one KV-head group, until about `target_pairs` visible pairs x heads."""
+    from paper_2602_24082_b200 import workloads as W
+    r = w.num_q_heads // w.num_kv_heads
+    order = sorted(range(len(w.rows)), key=lambda i: w.row_lengths()[i])
+    rows, pairs = [], 0
+    for i in order:
+        u = w.select_rows([i]).useful_pairs() * r
+        if rows and pairs + u > target_pairs:
+            break
+        rows.append(i)
+        pairs += u
+    nkv = 1
+    if len(rows) == len(w.rows):
+        nkv = int(max(1, min(w.num_kv_heads, target_pairs // max(pairs, 1))))
+    sub, stens, _, _ = W.slice_heads(w, tens, rows, list(range(nkv)))
+    return sub, stens, (f"rows {rows} (shortest first), KV heads 0..{nkv - 1} with their "
+                        f"{r * nkv} query heads, {sub.useful_pairs() * r * nkv} pair-heads")
+
+
+def time_oracle(sub, stens):
+    import oracle
+    t0 = time.perf_counter()
+    oracle.attn_fwd_bwd(sub.descriptors(), *stens, sub.softmax_scale)
+    dt = time.perf_counter() - t0
+    f, b = sub.useful_flops()
+    return (f + b) / dt / 1e12, dt, oracle.max_threads()
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = get_workload(args.config, 0)
+    tens = w.tensors()
+    sub, stens, what = oracle_sample(w, tens, target_pairs=5.0e7)
+    import oracle
+    oracle.build()
+    for _ in range(min(args.warmup, 1)):
+        time_oracle(sub, stens)
+    times, vals, cores = [], [], 1
+    for _ in range(args.steps):
+        v, dt, cores = time_oracle(sub, stens)
+        times.append(dt)
+        vals.append(v)
+    f, b = sub.useful_flops()
+    value = (f + b) * len(times) / sum(times) / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(times) / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": workload_config(w, args, sample=what),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def workload_config(w, args, **extra):
+    cfg = {
+        "workload": f"{args.config}: {w.name}, {len(w.rows)} rows, T={w.total_tokens} tokens, "
+                    f"Hq={w.num_q_heads}, Hkv={w.num_kv_heads}, D={w.head_dim}, "
+                    f"visible pairs U={w.useful_pairs()}",
+        "step": "pp_build_plan + pp_attn_fwd + pp_attn_bwd",
+        "l2": "flushed between timed steps (512 MiB write)",
+        "per_gpu_batch": "one batch of the recipe per GPU (seed differs per rank)",
+    }
+    cfg.update(extra)
+    return cfg
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2602_24082_b200 import binding as B
+    from paper_2602_24082_b200 import workloads as W
+    from paper_2602_24082_b200 import cost_model
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    B.lib()
+
+    w = get_workload(args.config, rank)
+    tens_cpu = w.tensors()
+    q, k, v, do = (x.to(dev) for x in tens_cpu)
+    desc = w.descriptors()
+    import numpy as np
+    desc_dev = [torch.from_numpy(np.ascontiguousarray(a)).to(dev) for a in desc]
+    T, Hq, Hkv, D = w.total_tokens, w.num_q_heads, w.num_kv_heads, w.head_dim
+    problem, _keep = B.make_problem(desc, Hq, Hkv, D, T, desc_dev)
+    plan_bytes, _, bwd_bytes = B.pp_plan_workspace_bytes(problem)
+    ws = torch.empty(plan_bytes, dtype=torch.uint8, device=dev)
+    o = torch.empty_like(q)
+    lse = torch.empty(Hq, T, dtype=torch.float32, device=dev)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    scale = w.softmax_scale
+    launches = {"n": 0}
+    plan_holder = {}
+
+    def step():
+        plan = B.pp_build_plan(desc, Hq, Hkv, D, T, dev, device_arrays=desc_dev, workspace=ws)
+        if "scratch" in plan_holder:
+            plan._bwd_scratch = plan_holder["scratch"]
+        B.pp_attn_fwd(plan, q, k, v, scale, o=o, lse=lse)
+        n = 4 + B.pp_last_launch_count()
+        B.pp_attn_bwd(plan, q, k, v, o, lse, do, scale, d_q=dq, d_k=dk, d_v=dv)
+        n += B.pp_last_launch_count()
+        plan_holder["scratch"] = plan.bwd_scratch()
+        plan_holder["plan"] = plan
+        return n
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps, count_launches=False, profile=False):
+        evs = []
+        kern = []
+        for _ in range(steps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            n = fn()
+            e1.record()
+            if count_launches:
+                launches["n"] += n
+            if profile:
+                torch.cuda.synchronize()
+                kern.append(B.pp_profile_read())
+            evs.append((e0, e1))
+        torch.cuda.synchronize()
+        return [a.elapsed_time(b) for a, b in evs], kern
+
+    # ---- warm-up, then the timed region
+    for _ in range(max(args.warmup, 3)):
+        flush.zero_()
+        step()
+    torch.cuda.synchronize()
+    st = plan_holder["plan"].status()
+    if st != (0, 0):
+        raise SystemExit(f"device status {st}")
+
+    B.pp_profile_enable(True)
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    ms, kern = timed(step, args.steps, count_launches=True, profile=True)
+    barrier()
+    clocks = sampler.stop()
+    B.pp_profile_enable(False)
+    total_ms = sum(ms)
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    f_flops, b_flops = w.useful_flops()
+    flops_all = float(f_flops + b_flops)
+    tokens_all = float(T)
+    if world > 1:
+        t = torch.tensor([flops_all, tokens_all], device=dev, dtype=torch.float64)
+        dist.all_reduce(t)
+        flops_all, tokens_all = float(t[0].item()), float(t[1].item())
+    value = flops_all / (ms_per_step * 1e-3) / 1e12
+
+    if args.quick:
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "ms_per_step": ms_per_step,
+                              "quick": True, "fwd_kernel_ms": statistics.mean(x[0] for x in kern),
+                              "bwd_kernel_ms": statistics.mean(x[1] for x in kern)}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- end to end through pp_attn_step_host: pinned host buffers, copies inside the timing
+    host = B.HostStep(w, dev)
+    hq, hk, hv, hdo = (x.pin_memory() for x in tens_cpu)
+    for _ in range(2):
+        host(hq, hk, hv, hdo)
+    torch.cuda.synchronize()
+    barrier()
+    e2e_ms, _ = timed(lambda: host(hq, hk, hv, hdo) and 0, max(3, min(args.steps, 10)))
+    barrier()
+    e2e_total = sum(e2e_ms) / len(e2e_ms)
+    if world > 1:
+        t = torch.tensor([e2e_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_total = float(t.item())
+    e2e_value = flops_all / (e2e_total * 1e-3) / 1e12
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (backward main), timed alone with CUDA events
+    peak, peak_sustained, peak_kind = peaks()
+    fwd_ms = statistics.mean(x[0] for x in kern)
+    bwd_ms = statistics.mean(x[1] for x in kern)
+    bwd_tflops = b_flops / (bwd_ms * 1e-3) / 1e12
+    fwd_tflops = f_flops / (fwd_ms * 1e-3) / 1e12
+    roofline = {"kernel": "bwd_kernel (dS/dQ/dK/dV main)", "bound": "tensor", "achieved": bwd_tflops,
+                "peak": peak, "unit": "TFLOP/s", "frac": bwd_tflops / peak, "peak_kind": f"of {peak_kind} (burst)",
+                "traffic": None, "avg_launch_ms": bwd_ms}
+    roofline_fwd = {"kernel": "fwd_kernel", "bound": "tensor", "achieved": fwd_tflops, "peak": peak,
+                    "unit": "TFLOP/s", "frac": fwd_tflops / peak, "avg_launch_ms": fwd_ms}
+
+    extra = {}
+    if world == 1:
+        # ---- the same kernels on the unpacked paired batch (each [x, y_k] its own sequence)
+        base = statistics.median(ms)
+        for padded in (True, False):
+            uw, gather = W.unpacked(w, padded=padded)
+            g = gather.to(dev)
+            uq, uk, uv, udo = (x.index_select(0, g).contiguous() for x in (q, k, v, do))
+            uplan = B.plan_for(uw, dev, desc_on_device=True)
+            uo, ulse = B.pp_attn_fwd(uplan, uq, uk, uv, scale)
+            B.pp_attn_bwd(uplan, uq, uk, uv, uo, ulse, udo, scale)
+
+            def ustep():
+                pl = B.pp_build_plan(uw.descriptors(), Hq, Hkv, D, uw.total_tokens, dev,
+                                     device_arrays=uplan._keep[1], workspace=uplan.workspace)
+                pl._bwd_scratch = uplan.bwd_scratch()
+                B.pp_attn_fwd(pl, uq, uk, uv, scale, o=uo, lse=ulse)
+                B.pp_attn_bwd(pl, uq, uk, uv, uo, ulse, udo, scale)
+                return 0
+
+            for _ in range(2):
+                ustep()
+            ums, _ = timed(ustep, max(3, min(args.steps, 10)))
+            key = "unpacked_padded" if padded else "unpacked_unpadded"
+            extra[key] = {"ms_per_step": statistics.median(ums), "tokens": uw.total_tokens,
+                          "speedup_of_packed": statistics.median(ums) / base,
+                          "useful_pair_ratio": uw.useful_pairs() / w.useful_pairs()}
+            del uq, uk, uv, udo, uo, ulse, uplan
+        grp = [(p, rs) for row in w.rows for (p, rs) in row]
+        extra["paper_cost_model_mean"] = {
+            "attention_cost_ratio": statistics.mean(cost_model.attention_cost_ratio(p, rs) for p, rs in grp),
+            "memory_ratio": statistics.mean(cost_model.memory_ratio(p, rs) for p, rs in grp)}
+
+    # ---- the CPU oracle beside it (rank 0, N = 1 only), on a bounded sample
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        sub, stens, what = oracle_sample(w, tens_cpu)
+        v_cpu, dt, cores = time_oracle(sub, stens)
+        cpu = {"value": v_cpu, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": what + f"; {dt:.1f} s"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": workload_config(w, args),
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": host.h2d_bytes,
+                "d2h_bytes_per_step": host.d2h_bytes, "ms_per_step": e2e_total,
+                "api": "pp_attn_step_host (pinned host buffers)"},
+        "gpu_launches": launches["n"],
+        "roofline": roofline,
+        "roofline_fwd": roofline_fwd,
+        "cpu_baseline": cpu,
+        "pct_of_peak": {"measured_burst": 100 * value / peak, "measured_sustained": 100 * value / peak_sustained,
+                        "nominal": 100 * value / NOMINAL_BF16_TFLOPS},
+        "tokens_per_s": tokens_all / (ms_per_step * 1e-3),
+        "ms_min_median": [min(ms), statistics.median(ms)],
+        "paper_context": PAPER_CONTEXT,
+    }
+    line.update(extra)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="config1")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--quick", action="store_true",
+                    help="timed steps only (no e2e, unpacked baseline or CPU leg): for profiler runs")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if args.steps == 100 and args.warmup == 5:
+            args.steps, args.warmup = 3, 1
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -123,8 +123,34 @@ int pp_attn_bwd(const pp_plan* plan, const void* q, const void* k, const void* v
                 const float* lse, const void* d_o, float softmax_scale, void* d_q, void* d_k,
                 void* d_v, void* d_scratch, size_t scratch_bytes, pp_stream_t stream);
 
-/* Kernel launches enqueued by the last pp_attn_fwd / pp_attn_bwd call of this thread. */
+/* Kernel launches enqueued by the last pp_attn_fwd / pp_attn_bwd / pp_attn_step_host call of
+ * this thread. */
 int pp_last_launch_count(void);
+
+/*
+ * One whole pass of the hot path on HOST buffers: copies Q, K, V, dO to the device, builds
+ * the plan from the host descriptors, runs forward and backward, and copies O, LSE, dQ, dK,
+ * dV back -- all enqueued on `stream`; the caller synchronises the stream before reading the
+ * outputs.  Host buffers should be page-locked for the copies to be asynchronous.  d_arena
+ * is caller-owned device memory of at least pp_step_host_arena_bytes (256-byte aligned); it
+ * holds the device copies, the plan workspace and the backward scratch.  `problem` must have
+ * desc_on_device == 0.  Same layouts and errors as the calls above.
+ */
+int pp_step_host_arena_bytes(const pp_problem* problem, size_t* arena_bytes);
+int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_k, const void* h_v,
+                      const void* h_do, float softmax_scale, void* h_o, float* h_lse, void* h_dq,
+                      void* h_dk, void* h_dv, void* d_arena, size_t arena_bytes,
+                      pp_stream_t stream);
+
+/*
+ * Kernel timing for benchmarks.  pp_profile_enable(1) makes pp_attn_fwd / pp_attn_bwd record
+ * CUDA events on the caller's stream directly around the forward kernel and around the
+ * backward main kernel; pp_profile_read returns the two durations (ms) of the most recent
+ * calls once that stream has been synchronised by the caller (PP_ERR_CUDA otherwise).
+ * pp_profile_enable(0) releases the events.
+ */
+int pp_profile_enable(int on);
+int pp_profile_read(float* fwd_kernel_ms, float* bwd_main_kernel_ms);
 
 const char* pp_error_string(int code);
 

@@ -22,7 +22,8 @@ _lib: Optional[ctypes.CDLL] = None
 
 EXPORTS = ["pp_plan_workspace_bytes", "pp_build_plan", "pp_plan_status", "pp_destroy_plan",
            "pp_plan_max_tiles", "pp_plan_read", "pp_attn_fwd", "pp_attn_bwd",
-           "pp_last_launch_count", "pp_error_string"]
+           "pp_last_launch_count", "pp_error_string", "pp_step_host_arena_bytes",
+           "pp_attn_step_host", "pp_profile_enable", "pp_profile_read"]
 
 
 class PPError(RuntimeError):
@@ -66,6 +67,10 @@ def lib() -> ctypes.CDLL:
         L.pp_plan_read.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         L.pp_attn_fwd.argtypes = [vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, sz, vp]
         L.pp_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, sz, vp]
+        L.pp_step_host_arena_bytes.argtypes = [vp, vp]
+        L.pp_attn_step_host.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.pp_profile_enable.argtypes = [ctypes.c_int]
+        L.pp_profile_read.argtypes = [vp, vp]
         _lib = L
     return _lib
 
@@ -154,15 +159,21 @@ def pp_plan_workspace_bytes(problem: _Problem) -> Tuple[int, int, int]:
 
 
 def pp_build_plan(desc: Sequence[np.ndarray], num_q_heads: int, num_kv_heads: int, head_dim: int,
-                  total_tokens: int, device: str = "cuda:0", desc_on_device: bool = False) -> Plan:
+                  total_tokens: int, device: str = "cuda:0", desc_on_device: bool = False,
+                  device_arrays: Optional[Sequence[torch.Tensor]] = None,
+                  workspace: Optional[torch.Tensor] = None) -> Plan:
+    """Builds a plan.  ``device_arrays`` (int32 CUDA tensors) and ``workspace`` (uint8 CUDA
+    tensor of at least the queried size) let a caller re-plan every step without allocating."""
     if not torch.cuda.is_available():
         raise RuntimeError("pp_build_plan needs a CUDA device (there is no CPU fallback)")
-    dev_arrays = None
-    if desc_on_device:
+    dev_arrays = device_arrays
+    if desc_on_device and dev_arrays is None:
         dev_arrays = [torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device) for a in desc]
     problem, keep = make_problem(desc, num_q_heads, num_kv_heads, head_dim, total_tokens, dev_arrays)
     sizes = pp_plan_workspace_bytes(problem)
-    ws = torch.empty(sizes[0], dtype=torch.uint8, device=device)
+    ws = workspace if workspace is not None else torch.empty(sizes[0], dtype=torch.uint8, device=device)
+    if ws.numel() < sizes[0]:
+        raise ValueError("workspace too small")
     handle = ctypes.c_void_p(0)
     with torch.cuda.device(ws.device):
         _check(lib().pp_build_plan(ctypes.byref(problem), ws.data_ptr(), sizes[0], _stream(),
@@ -216,6 +227,61 @@ def pp_attn_bwd(plan: Plan, q, k, v, o, lse, d_o, softmax_scale: float, d_q=None
                                  d_q.data_ptr(), d_k.data_ptr(), d_v.data_ptr(), scratch.data_ptr(),
                                  scratch.numel(), _stream()), "pp_attn_bwd")
     return d_q, d_k, d_v
+
+
+def pp_step_host_arena_bytes(problem: _Problem) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().pp_step_host_arena_bytes(ctypes.byref(problem), ctypes.byref(n)),
+           "pp_step_host_arena_bytes")
+    return n.value
+
+
+class HostStep:
+    """pp_attn_step_host on page-locked host tensors: one whole pass (H2D copies, plan,
+    forward, backward, D2H copies) enqueued on the current stream."""
+
+    def __init__(self, workload, device: str = "cuda:0"):
+        if not torch.cuda.is_available():
+            raise RuntimeError("pp_attn_step_host needs a CUDA device (there is no CPU fallback)")
+        w = workload
+        self.scale = w.softmax_scale
+        self.problem, self._keep = make_problem(w.descriptors(), w.num_q_heads, w.num_kv_heads,
+                                                w.head_dim, w.total_tokens)
+        self.arena = torch.empty(pp_step_host_arena_bytes(self.problem), dtype=torch.uint8,
+                                 device=device)
+        T, Hq, Hkv, D = w.total_tokens, w.num_q_heads, w.num_kv_heads, w.head_dim
+        pin = lambda *shape, dtype=torch.bfloat16: torch.empty(*shape, dtype=dtype).pin_memory()
+        self.o, self.dq = pin(T, Hq, D), pin(T, Hq, D)
+        self.dk, self.dv = pin(T, Hkv, D), pin(T, Hkv, D)
+        self.lse = pin(Hq, T, dtype=torch.float32)
+        self.h2d_bytes = 2 * D * T * (2 * Hq + 2 * Hkv)
+        self.d2h_bytes = 2 * D * T * (2 * Hq + 2 * Hkv) + 4 * Hq * T
+
+    def __call__(self, q, k, v, d_o):
+        """q, k, v, d_o: page-locked CPU bf16 tensors.  Results land in self.o, .lse, .dq, .dk,
+        .dv once the current stream has been synchronised."""
+        for t in (q, k, v, d_o):
+            if t.is_cuda or not t.is_contiguous() or t.dtype != torch.bfloat16:
+                raise ValueError("pp_attn_step_host takes contiguous CPU bf16 tensors")
+        with torch.cuda.device(self.arena.device):
+            _check(lib().pp_attn_step_host(ctypes.byref(self.problem), q.data_ptr(), k.data_ptr(),
+                                           v.data_ptr(), d_o.data_ptr(), float(self.scale),
+                                           self.o.data_ptr(), self.lse.data_ptr(), self.dq.data_ptr(),
+                                           self.dk.data_ptr(), self.dv.data_ptr(),
+                                           self.arena.data_ptr(), self.arena.numel(), _stream()),
+                   "pp_attn_step_host")
+        return self.o, self.lse, self.dq, self.dk, self.dv
+
+
+def pp_profile_enable(on: bool):
+    _check(lib().pp_profile_enable(1 if on else 0), "pp_profile_enable")
+
+
+def pp_profile_read() -> Tuple[float, float]:
+    """(forward kernel ms, backward main kernel ms) of the latest calls; sync the stream first."""
+    a, b = ctypes.c_float(0), ctypes.c_float(0)
+    _check(lib().pp_profile_read(ctypes.byref(a), ctypes.byref(b)), "pp_profile_read")
+    return a.value, b.value
 
 
 def pp_last_launch_count() -> int:

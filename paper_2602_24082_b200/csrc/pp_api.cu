@@ -199,6 +199,68 @@ int pp_attn_bwd(const pp_plan* plan, const void* q, const void* k, const void* v
 
 int pp_last_launch_count(void) { return g_last_launches; }
 
+int pp_step_host_arena_bytes(const pp_problem* problem, size_t* arena_bytes) {
+  int rc = check_problem_shape(problem);
+  if (rc) return rc;
+  if (!arena_bytes) return PP_ERR_INVALID_ARG;
+  *arena_bytes = pp::step_arena_layout(*problem).total;
+  return PP_OK;
+}
+
+int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_k, const void* h_v,
+                      const void* h_do, float softmax_scale, void* h_o, float* h_lse, void* h_dq,
+                      void* h_dk, void* h_dv, void* d_arena, size_t arena_bytes,
+                      pp_stream_t stream) {
+  g_last_launches = 0;
+  int rc = check_problem_shape(problem);
+  if (rc) return rc;
+  if (problem->desc_on_device) return PP_ERR_INVALID_ARG;
+  if (!h_q || !h_k || !h_v || !h_do || !h_o || !h_lse || !h_dq || !h_dk || !h_dv || !d_arena)
+    return PP_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(d_arena) & 255) return PP_ERR_ALIGNMENT;
+  pp::StepArena a = pp::step_arena_layout(*problem);
+  if (arena_bytes < a.total) return PP_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  char* base = static_cast<char*>(d_arena);
+  const size_t T = problem->total_tokens, D = problem->head_dim;
+  const size_t qb = T * problem->num_q_heads * D * 2, kb = T * problem->num_kv_heads * D * 2;
+  const size_t lb = T * problem->num_q_heads * 4;
+  bool ok = cudaMemcpyAsync(base + a.q, h_q, qb, cudaMemcpyHostToDevice, s) == cudaSuccess &&
+            cudaMemcpyAsync(base + a.k, h_k, kb, cudaMemcpyHostToDevice, s) == cudaSuccess &&
+            cudaMemcpyAsync(base + a.v, h_v, kb, cudaMemcpyHostToDevice, s) == cudaSuccess &&
+            cudaMemcpyAsync(base + a.d_o, h_do, qb, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  if (!ok) return PP_ERR_CUDA;
+  pp_plan* plan = nullptr;
+  rc = pp_build_plan(problem, base + a.plan, a.scratch - a.plan, stream, &plan);
+  if (rc) return rc;
+  int launches = 4;
+  rc = pp_attn_fwd(plan, base + a.q, base + a.k, base + a.v, softmax_scale, base + a.o,
+                   reinterpret_cast<float*>(base + a.lse), nullptr, 0, stream);
+  launches += g_last_launches;
+  if (rc == PP_OK) {
+    rc = pp_attn_bwd(plan, base + a.q, base + a.k, base + a.v, base + a.o,
+                     reinterpret_cast<float*>(base + a.lse), base + a.d_o, softmax_scale,
+                     base + a.dq, base + a.dk, base + a.dv, base + a.scratch, a.total - a.scratch,
+                     stream);
+    launches += g_last_launches;
+  }
+  pp_destroy_plan(plan);
+  g_last_launches = launches;
+  if (rc) return rc;
+  ok = cudaMemcpyAsync(h_o, base + a.o, qb, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
+       cudaMemcpyAsync(h_lse, base + a.lse, lb, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
+       cudaMemcpyAsync(h_dq, base + a.dq, qb, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
+       cudaMemcpyAsync(h_dk, base + a.dk, kb, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
+       cudaMemcpyAsync(h_dv, base + a.dv, kb, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  return ok ? PP_OK : PP_ERR_CUDA;
+}
+
+int pp_profile_enable(int on) { return pp::profile_enable(on != 0) ? PP_OK : PP_ERR_CUDA; }
+
+int pp_profile_read(float* fwd_kernel_ms, float* bwd_main_kernel_ms) {
+  return pp::profile_read(fwd_kernel_ms, bwd_main_kernel_ms) ? PP_OK : PP_ERR_CUDA;
+}
+
 const char* pp_error_string(int code) {
   switch (code) {
     case PP_OK: return "ok";

@@ -318,7 +318,13 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
       static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse,
       const_cast<float*>(prm.delta), const_cast<float*>(prm.lse2), int(T), int(Hq));
   dim3 grid(unsigned(plan->max_tiles) * unsigned(pb.num_kv_heads));
+  ProfileEvents& ev = profile_events();
+  if (ev.on) cudaEventRecord(ev.bwd0, stream);
   kern<<<grid, kBwdThreads, BwdSmem<D>::kTotal, stream>>>(tq, tk, tv, tdo, prm);
+  if (ev.on) {
+    cudaEventRecord(ev.bwd1, stream);
+    ev.bwd_valid = true;
+  }
   const size_t n4 = T * Hq * D / 4;
   unsigned fb = unsigned(std::min<size_t>((n4 + 255) / 256, 148 * 16));
   bwd_finalize_kernel<<<fb, 256, 0, stream>>>(reinterpret_cast<const float4*>(prm.dq_acc),

@@ -222,7 +222,13 @@ cudaError_t launch_fwd_t(const pp_plan* plan, const CUtensorMap& tq, const CUten
     configured = true;
   }
   dim3 grid(unsigned(plan->max_tiles) * unsigned(plan->prob.num_q_heads));
+  ProfileEvents& ev = profile_events();
+  if (ev.on) cudaEventRecord(ev.fwd0, stream);
   kern<<<grid, kFwdThreads, FwdSmem<D>::kTotal, stream>>>(tq, tk, tv, prm);
+  if (ev.on) {
+    cudaEventRecord(ev.fwd1, stream);
+    ev.fwd_valid = true;
+  }
   return cudaGetLastError();
 }
 

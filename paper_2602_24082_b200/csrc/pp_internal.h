@@ -100,6 +100,35 @@ inline BwdScratch bwd_scratch_layout(const pp_problem& p) {
   return s;
 }
 
+// Device arena of pp_attn_step_host: inputs, outputs, plan workspace, backward scratch.
+struct StepArena {
+  size_t q, k, v, d_o, o, lse, dq, dk, dv, plan, scratch, total;
+};
+inline StepArena step_arena_layout(const pp_problem& p) {
+  StepArena a{};
+  const size_t T = p.total_tokens, D = p.head_dim;
+  const size_t qb = T * p.num_q_heads * D * 2, kb = T * p.num_kv_heads * D * 2;
+  size_t off = 0;
+  auto take = [&](size_t n) { size_t o = off; off = align_up(off + n, 256); return o; };
+  a.q = take(qb); a.k = take(kb); a.v = take(kb); a.d_o = take(qb);
+  a.o = take(qb); a.lse = take(T * p.num_q_heads * 4);
+  a.dq = take(qb); a.dk = take(kb); a.dv = take(kb);
+  a.plan = take(plan_layout(p).total);
+  a.scratch = take(bwd_scratch_layout(p).total);
+  a.total = off;
+  return a;
+}
+
+// Optional event pairs around the forward kernel and the backward main kernel.
+struct ProfileEvents {
+  bool on = false;
+  cudaEvent_t fwd0 = nullptr, fwd1 = nullptr, bwd0 = nullptr, bwd1 = nullptr;
+  bool fwd_valid = false, bwd_valid = false;
+};
+ProfileEvents& profile_events();
+bool profile_enable(bool on);
+bool profile_read(float* fwd_ms, float* bwd_ms);
+
 // launchers (defined in the .cu files); all return a cudaError_t
 cudaError_t launch_plan(const pp_plan* plan, cudaStream_t stream);
 cudaError_t launch_fwd(const pp_plan* plan, const void* q, const void* k, const void* v, float scale,

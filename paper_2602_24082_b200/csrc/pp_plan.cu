@@ -199,6 +199,36 @@ __global__ void plan_order_kernel(PlanPtrs p) {
 
 }  // namespace
 
+ProfileEvents& profile_events() {
+  static ProfileEvents ev;
+  return ev;
+}
+
+bool profile_enable(bool on) {
+  ProfileEvents& ev = profile_events();
+  if (on == ev.on) return true;
+  if (on) {
+    bool ok = cudaEventCreate(&ev.fwd0) == cudaSuccess && cudaEventCreate(&ev.fwd1) == cudaSuccess &&
+              cudaEventCreate(&ev.bwd0) == cudaSuccess && cudaEventCreate(&ev.bwd1) == cudaSuccess;
+    ev.on = ok;
+    ev.fwd_valid = ev.bwd_valid = false;
+    return ok;
+  }
+  cudaEventDestroy(ev.fwd0); cudaEventDestroy(ev.fwd1);
+  cudaEventDestroy(ev.bwd0); cudaEventDestroy(ev.bwd1);
+  ev = ProfileEvents();
+  return true;
+}
+
+bool profile_read(float* fwd_ms, float* bwd_ms) {
+  ProfileEvents& ev = profile_events();
+  if (!ev.on) return false;
+  bool ok = true;
+  if (fwd_ms) ok = ok && ev.fwd_valid && cudaEventElapsedTime(fwd_ms, ev.fwd0, ev.fwd1) == cudaSuccess;
+  if (bwd_ms) ok = ok && ev.bwd_valid && cudaEventElapsedTime(bwd_ms, ev.bwd0, ev.bwd1) == cudaSuccess;
+  return ok;
+}
+
 cudaError_t launch_plan(const pp_plan* plan, cudaStream_t stream) {
   PlanPtrs p;
   char* ws = plan->ws;

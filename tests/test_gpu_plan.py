@@ -1,0 +1,93 @@
+"""The device-built plan against a host re-derivation from the dense mask."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2602_24082_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+CASES = [
+    W.config0(),
+    W.Workload("ragged", [[(257, (5, 128, 31))], [(1, (1, 300))]], 4, 2, 128, seed=4),
+    W.Workload("groups", [[(97, (64, 200)), (128, (128, 128)), (3, (2, 1))], [(700, (1,))]], 2, 2, 64, seed=5),
+    W.config3(),
+]
+
+
+def _global_mask(w):
+    T = w.total_tokens
+    m = np.zeros((T, T), dtype=bool)
+    offs = w.row_offsets()
+    for r in range(len(w.rows)):
+        m[offs[r]:offs[r + 1], offs[r]:offs[r + 1]] = oracle.dense_mask(w.descriptors(), r)
+    return m
+
+
+@pytest.mark.parametrize("w", CASES, ids=lambda w: w.name)
+@pytest.mark.parametrize("desc_on_device", [False, True], ids=["hostdesc", "devdesc"])
+def test_plan_matches_dense_mask(w, desc_on_device):
+    from paper_2602_24082_b200 import binding as B
+    plan = B.plan_for(w, desc_on_device=desc_on_device)
+    assert plan.status() == (0, 0)
+    tiles, fwd_order, bwd_order, key_end = plan.read()
+    mask = _global_mask(w)
+    T = w.total_tokens
+    # tiles partition the tokens, never straddle a segment
+    segs = w.segments()
+    covered = np.zeros(T, dtype=int)
+    expect_tiles = sum((l + 127) // 128 for (_, l, *_rest) in segs)
+    assert len(tiles) == expect_tiles
+    for (start, ln, k0s, k0l, k1s, k1l, vis_end, work) in tiles.tolist():
+        assert 1 <= ln <= 128
+        covered[start:start + ln] += 1
+        seg = [s for s in segs if s[0] <= start < s[0] + s[1]][0]
+        assert start + ln <= seg[0] + seg[1] and (start - seg[0]) % 128 == 0
+        # forward view: every row of the tile sees exactly kv0 U kv1 (FULL, no masked pair)
+        # plus the causal part of its own tile (DIAG); nothing else (siblings are skipped)
+        rows = mask[start:start + ln]
+        want = np.zeros((ln, T), dtype=bool)
+        want[:, k0s:k0s + k0l] = True
+        want[:, k1s:k1s + k1l] = True
+        want[:, start:start + ln] = np.tril(np.ones((ln, ln), dtype=bool))
+        assert np.array_equal(rows, want)
+        assert work == (k0l + 127) // 128 + (k1l + 127) // 128 + 1
+        # backward view: the queries that see these keys are exactly [start, vis_end),
+        # fully below the tile, causally inside it
+        cols = mask[:, start:start + ln]
+        wantc = np.zeros((T, ln), dtype=bool)
+        wantc[start:start + ln] = np.tril(np.ones((ln, ln), dtype=bool))
+        wantc[start + ln:vis_end] = True
+        assert np.array_equal(cols, wantc)
+    assert (covered == 1).all()
+    # column form of the mask: key j is visible to queries [j, key_end[j])
+    for j in range(0, T, max(1, T // 997)):
+        seen = np.nonzero(mask[:, j])[0]
+        assert seen[0] == j and seen[-1] + 1 == key_end[j] and len(seen) == key_end[j] - j
+    # orders are permutations, longest work first
+    n = len(tiles)
+    assert sorted(fwd_order.tolist()) == list(range(n)) and sorted(bwd_order.tolist()) == list(range(n))
+    fw = tiles[fwd_order, 7]
+    assert (np.diff(fw) <= 0).all()
+    bw = 1 + (tiles[:, 6] - tiles[:, 0] - tiles[:, 1] + 127) // 128
+    assert (np.diff(bw[bwd_order]) <= 0).all()
+
+
+def test_device_side_validation_reports_status():
+    from paper_2602_24082_b200 import binding as B
+    w = W.Workload("bad", [[(5, (2, 4))], [(3, (1, 2))]], 2, 1, 64, seed=0)
+    rgo, gpl, gro, rl = w.descriptors()
+    bad_rl = rl.copy(); bad_rl[2] = 0
+    plan = B.pp_build_plan((rgo, gpl, gro, bad_rl), 2, 1, 64, w.total_tokens, desc_on_device=True)
+    st, det = plan.status()
+    assert st == 1 and det == len(gpl) + 2
+    bad_rl = rl.copy(); bad_rl[0] += 3
+    plan = B.pp_build_plan((rgo, gpl, gro, bad_rl), 2, 1, 64, w.total_tokens, desc_on_device=True)
+    assert plan.status() == (2, w.total_tokens + 3)
+    # kernels given a failed plan do nothing and report nothing new
+    import torch
+    q, k, v, do = (x.cuda() for x in w.tensors())
+    o = torch.full_like(q, 3.0)
+    B.pp_attn_fwd(plan, q, k, v, 0.125, o=o)
+    torch.cuda.synchronize()
+    assert (o == 3.0).all()
