@@ -42,7 +42,8 @@ enum pp_status {
   PP_ERR_WORKSPACE_TOO_SMALL = -3, /* plan workspace or scratch smaller than the size query says */
   PP_ERR_ALIGNMENT = -4,           /* a tensor base pointer is not 16-byte aligned */
   PP_ERR_CUDA = -5,                /* a CUDA runtime / driver call failed */
-  PP_ERR_PLAN_STATUS = -6          /* device-side validation failed or a bounded wait expired */
+  PP_ERR_PLAN_STATUS = -6,         /* device-side validation failed or a bounded wait expired */
+  PP_ERR_STATIC_SCRATCH_LIMIT = -7 /* pp_attn_bwd_noalloc: problem larger than its built-in scratch */
 };
 
 /*
@@ -122,6 +123,36 @@ int pp_attn_fwd(const pp_plan* plan, const void* q, const void* k, const void* v
 int pp_attn_bwd(const pp_plan* plan, const void* q, const void* k, const void* v, const void* o,
                 const float* lse, const void* d_o, float softmax_scale, void* d_q, void* d_k,
                 void* d_v, void* d_scratch, size_t scratch_bytes, pp_stream_t stream);
+
+/*
+ * pp_attn_bwd for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this is a packaging variant of the backward above, not a different computation.)
+ *
+ * Some callers have no way to hand the library a scratch buffer: an extension loaded into a
+ * host application that owns the whole device heap and gives plug-ins none of it, a step
+ * running after every byte has been committed to other tenants, or a latency-critical loop
+ * in which cudaMalloc / cudaFree are forbidden because they may synchronise the device.  For
+ * them the backward's scratch (fp32 dQ accumulator, Delta, scaled LSE) lives in an array that
+ * is part of the library image.  This entry point calls no cudaMalloc, cudaFree or other
+ * allocating routine; the caller still passes every input and output tensor.
+ *
+ *  - Limit: the scratch pp_plan_workspace_bytes reports for the plan's problem must not exceed
+ *    pp_attn_bwd_noalloc_max_bytes (32 MiB, i.e. about T * Hq * D <= 8.2 M elements);
+ *    larger problems are rejected with PP_ERR_STATIC_SCRATCH_LIMIT and nothing is launched.
+ *  - Cost: every GPU on which the library is loaded holds those 32 MiB until the process exits.
+ *  - The first call on each device looks up the array's device address (with that device
+ *    current).  Make that first call before any stream capture begins.
+ *  - All calls on a device share the one array, and it keeps the previous call's contents.
+ *    Each call clears the part that must start at zero (the dQ accumulator) and rewrites
+ *    the rest, so back-to-back calls on ONE stream are safe; calls that can overlap on the
+ *    GPU (different streams, different host threads without ordering) race on it and give
+ *    wrong gradients.
+ * Results, layouts and the other errors are those of pp_attn_bwd.
+ */
+int pp_attn_bwd_noalloc_max_bytes(size_t* bytes);
+int pp_attn_bwd_noalloc(const pp_plan* plan, const void* q, const void* k, const void* v,
+                        const void* o, const float* lse, const void* d_o, float softmax_scale,
+                        void* d_q, void* d_k, void* d_v, pp_stream_t stream);
 
 /* Kernel launches enqueued by the last pp_attn_fwd / pp_attn_bwd / pp_attn_step_host call of
  * this thread. */

@@ -23,7 +23,8 @@ _lib: Optional[ctypes.CDLL] = None
 EXPORTS = ["pp_plan_workspace_bytes", "pp_build_plan", "pp_plan_status", "pp_destroy_plan",
            "pp_plan_max_tiles", "pp_plan_read", "pp_attn_fwd", "pp_attn_bwd",
            "pp_last_launch_count", "pp_error_string", "pp_step_host_arena_bytes",
-           "pp_attn_step_host", "pp_profile_enable", "pp_profile_read"]
+           "pp_attn_step_host", "pp_profile_enable", "pp_profile_read",
+           "pp_attn_bwd_noalloc", "pp_attn_bwd_noalloc_max_bytes"]
 
 
 class PPError(RuntimeError):
@@ -69,6 +70,8 @@ def lib() -> ctypes.CDLL:
         L.pp_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, sz, vp]
         L.pp_step_host_arena_bytes.argtypes = [vp, vp]
         L.pp_attn_step_host.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.pp_attn_bwd_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
+        L.pp_attn_bwd_noalloc_max_bytes.argtypes = [vp]
         L.pp_profile_enable.argtypes = [ctypes.c_int]
         L.pp_profile_read.argtypes = [vp, vp]
         _lib = L
@@ -226,6 +229,32 @@ def pp_attn_bwd(plan: Plan, q, k, v, o, lse, d_o, softmax_scale: float, d_q=None
                                  o.data_ptr(), lse.data_ptr(), d_o.data_ptr(), float(softmax_scale),
                                  d_q.data_ptr(), d_k.data_ptr(), d_v.data_ptr(), scratch.data_ptr(),
                                  scratch.numel(), _stream()), "pp_attn_bwd")
+    return d_q, d_k, d_v
+
+
+def pp_attn_bwd_noalloc_max_bytes() -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().pp_attn_bwd_noalloc_max_bytes(ctypes.byref(n)), "pp_attn_bwd_noalloc_max_bytes")
+    return n.value
+
+
+def pp_attn_bwd_noalloc(plan: Plan, q, k, v, o, lse, d_o, softmax_scale: float, d_q, d_k, d_v):
+    """Backward for callers that must not allocate: the scratch is an array inside the
+    library (32 MiB per GPU), so the outputs have to be passed in and nothing is allocated
+    here either.  Problems whose scratch exceeds pp_attn_bwd_noalloc_max_bytes() raise
+    PPError(-7).  Calls on one stream may follow each other; overlapping calls race."""
+    p = plan.problem
+    T, Hq, Hkv, D = p.total_tokens, p.num_q_heads, p.num_kv_heads, p.head_dim
+    for t, shape, name in ((q, (T, Hq, D), "q"), (k, (T, Hkv, D), "k"), (v, (T, Hkv, D), "v"),
+                           (o, (T, Hq, D), "o"), (d_o, (T, Hq, D), "d_o"), (d_q, (T, Hq, D), "d_q"),
+                           (d_k, (T, Hkv, D), "d_k"), (d_v, (T, Hkv, D), "d_v")):
+        _chk(t, shape, torch.bfloat16, name)
+    _chk(lse, (Hq, T), torch.float32, "lse")
+    with torch.cuda.device(q.device):
+        _check(lib().pp_attn_bwd_noalloc(plan.handle, q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                         o.data_ptr(), lse.data_ptr(), d_o.data_ptr(),
+                                         float(softmax_scale), d_q.data_ptr(), d_k.data_ptr(),
+                                         d_v.data_ptr(), _stream()), "pp_attn_bwd_noalloc")
     return d_q, d_k, d_v
 
 

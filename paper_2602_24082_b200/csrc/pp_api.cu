@@ -197,6 +197,28 @@ int pp_attn_bwd(const pp_plan* plan, const void* q, const void* k, const void* v
   return e == cudaSuccess ? PP_OK : (e == cudaErrorNotSupported ? PP_ERR_UNSUPPORTED : PP_ERR_CUDA);
 }
 
+int pp_attn_bwd_noalloc_max_bytes(size_t* bytes) {
+  if (!bytes) return PP_ERR_INVALID_ARG;
+  *bytes = pp::kStaticScratchBytes;
+  return PP_OK;
+}
+
+int pp_attn_bwd_noalloc(const pp_plan* plan, const void* q, const void* k, const void* v,
+                        const void* o, const float* lse, const void* d_o, float softmax_scale,
+                        void* d_q, void* d_k, void* d_v, pp_stream_t stream) {
+  g_last_launches = 0;
+  if (!plan || !q || !k || !v || !o || !lse || !d_o || !d_q || !d_k || !d_v)
+    return PP_ERR_INVALID_ARG;
+  if (!(softmax_scale > 0.f) || softmax_scale > 1e30f) return PP_ERR_INVALID_ARG;
+  if (plan->bwd_scratch > pp::kStaticScratchBytes) return PP_ERR_STATIC_SCRATCH_LIMIT;
+  const void* ptrs[] = {q, k, v, o, lse, d_o, d_q, d_k, d_v};
+  for (const void* p : ptrs)
+    if (!aligned16(p)) return PP_ERR_ALIGNMENT;
+  cudaError_t e = pp::launch_bwd_static(plan, q, k, v, o, lse, d_o, softmax_scale, d_q, d_k, d_v,
+                                        reinterpret_cast<cudaStream_t>(stream), &g_last_launches);
+  return e == cudaSuccess ? PP_OK : (e == cudaErrorNotSupported ? PP_ERR_UNSUPPORTED : PP_ERR_CUDA);
+}
+
 int pp_last_launch_count(void) { return g_last_launches; }
 
 int pp_step_host_arena_bytes(const pp_problem* problem, size_t* arena_bytes) {
@@ -270,6 +292,9 @@ const char* pp_error_string(int code) {
     case PP_ERR_ALIGNMENT: return "pointer not sufficiently aligned";
     case PP_ERR_CUDA: return "CUDA call failed";
     case PP_ERR_PLAN_STATUS: return "device-side validation failed or a bounded wait expired";
+    case PP_ERR_STATIC_SCRATCH_LIMIT:
+      return "problem needs more backward scratch than the 32 MiB built into the library; "
+             "use pp_attn_bwd with caller-provided scratch";
     default: return "unknown error";
   }
 }

@@ -13,6 +13,7 @@
 //                it is added into an fp32 accumulator with vector reductions.
 //   finalize   : dQ = bf16(scale * accumulator)
 #include <algorithm>
+#include <mutex>
 
 #include "pp_dev.cuh"
 
@@ -364,6 +365,45 @@ cudaError_t launch_bwd(const pp_plan* plan, const void* q, const void* k, const 
   return pb.head_dim == 128
              ? launch_bwd_t<128>(plan, o, lse, d_o, dq, tq, tk, tv, tdo, prm, stream, launches)
              : launch_bwd_t<64>(plan, o, lse, d_o, dq, tq, tk, tv, tdo, prm, stream, launches);
+}
+
+// ---------------------------------------------------------------- built-in scratch
+// Backward scratch for callers that cannot allocate device memory (pp_attn_bwd_noalloc).
+// The array is part of the library image: every device that loads the library holds
+// kStaticScratchBytes until the process exits, and every call on a device shares it.
+static __device__ __align__(256) unsigned char g_static_bwd_scratch[kStaticScratchBytes];
+
+// In host code `g_static_bwd_scratch` is only a stand-in for the symbol, not a device
+// address, so the address is looked up once per device (with that device current) and kept.
+static cudaError_t static_scratch_address(void** out) {
+  constexpr int kMaxDevices = 64;
+  static std::mutex mu;
+  static void* ptrs[kMaxDevices] = {};
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!ptrs[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_bwd_scratch);
+    if (e != cudaSuccess) return e;
+    if (!p) return cudaErrorInvalidSymbol;
+    ptrs[dev] = p;
+  }
+  *out = ptrs[dev];
+  return cudaSuccess;
+}
+
+cudaError_t launch_bwd_static(const pp_plan* plan, const void* q, const void* k, const void* v,
+                              const void* o, const float* lse, const void* d_o, float scale,
+                              void* dq, void* dk, void* dv, cudaStream_t stream, int* launches) {
+  void* scratch = nullptr;
+  cudaError_t e = static_scratch_address(&scratch);
+  if (e != cudaSuccess) return e;
+  // launch_bwd zeroes the fp32 dQ accumulator inside the scratch on every call and rewrites
+  // Delta and the scaled LSE, so nothing of an earlier call's contents is read.
+  return launch_bwd(plan, q, k, v, o, lse, d_o, scale, dq, dk, dv, scratch, stream, launches);
 }
 
 }  // namespace pp

@@ -137,4 +137,10 @@ cudaError_t launch_bwd(const pp_plan* plan, const void* q, const void* k, const 
                        const void* o, const float* lse, const void* d_o, float scale, void* dq,
                        void* dk, void* dv, void* scratch, cudaStream_t stream, int* launches);
 
+// Size of the scratch array built into the library image for pp_attn_bwd_noalloc.
+constexpr size_t kStaticScratchBytes = size_t(32) << 20;
+cudaError_t launch_bwd_static(const pp_plan* plan, const void* q, const void* k, const void* v,
+                              const void* o, const float* lse, const void* d_o, float scale,
+                              void* dq, void* dk, void* dv, cudaStream_t stream, int* launches);
+
 }  // namespace pp
