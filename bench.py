@@ -291,8 +291,11 @@ def run_ours(args):
     if args.quick:
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "ms_per_step": ms_per_step,
-                              "quick": True, "fwd_kernel_ms": statistics.mean(x[0] for x in kern),
-                              "bwd_kernel_ms": statistics.mean(x[1] for x in kern)}))
+                              "quick": True, "workload": w.name,
+                              "fwd_kernel_ms": statistics.mean(x[0] for x in kern),
+                              "bwd_kernel_ms": statistics.mean(x[1] for x in kern),
+                              "fwd_tflops": f_flops / statistics.mean(x[0] for x in kern) / 1e9,
+                              "bwd_tflops": b_flops / statistics.mean(x[1] for x in kern) / 1e9}))
         if world > 1:
             dist.destroy_process_group()
         return

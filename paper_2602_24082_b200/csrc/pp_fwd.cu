@@ -1,12 +1,21 @@
 // Forward kernel: O = softmax(mask(scale Q K^T)) V and LSE over the plan's visible tiles.
 //
-// One CTA per (query tile, query head).  TMA stages Q once and K/V per key tile in 128-byte
-// swizzled shared memory; tcgen05.mma accumulates S = Q K^T and O += P V in tensor memory
-// (fp32); each of the 128 threads owns one query row (= one TMEM lane) for the online
-// softmax, so row maxima and sums need no cross-thread traffic.  P is rounded to bf16 and
-// written back into tensor memory, over the columns S occupied, where the second MMA reads
-// it as its A operand.  Two CTAs fit per SM (256 TMEM columns, 96 KB shared memory each), so
-// one CTA's softmax overlaps the other's MMAs.
+// Persistent, warp-specialised CTA (one per SM):
+//   warp 0      TMA producer: Q tiles of the unit's two query heads, then the K / V tiles of
+//               every visible key tile through two-stage rings
+//   warp 1      MMA issuer (one thread): S = Q K^T and O += P V with tcgen05.mma, fp32 in TMEM
+//   warps 2-5   softmax warpgroup of slot 0: thread = query row = TMEM lane
+//   warps 6-9   softmax warpgroup of slot 1
+// A work unit is (query tile, KV head, pair of query heads of that KV head): both slots see
+// the same keys and the same mask, so every K / V tile staged in shared memory feeds two
+// S tiles.  While one slot's warpgroup does its exponentials the tensor core works on the
+// other slot (order: PV_0(j), QK_0(j+1), PV_1(j), QK_1(j+1), ...).  P (bf16) overwrites the
+// first 64 columns of its S tile in tensor memory and is the A operand of the second MMA; V is
+// its MN-major B operand straight from the TMA layout.  O is rescaled lazily: only when a
+// row's running maximum grew by more than 2^8 since the value used for scaling.
+// TMEM: S0 | S1 | O0 | O1, 128 columns each.
+#include <algorithm>
+
 #include "pp_dev.cuh"
 
 namespace pp {
@@ -22,43 +31,107 @@ struct FwdParams {
   float scale_log2;  // softmax scale * log2(e)
 };
 
-constexpr int kFwdThreads = 128;
-constexpr uint32_t kFwdTmemCols = 256;  // [0,128): S then P (bf16, 64 columns); [128, 128+D): O
+constexpr int kFwdThreads = 320;
+constexpr uint32_t kFwdTmemCols = 512;
+constexpr float kRescaleThreshold = 8.f;  // log2 units
+
+enum FwdBar : int {
+  kQFull = 0,   // [2] per slot
+  kQEmpty = 2,  // [2]
+  kKFull = 4,   // [2] per stage
+  kKEmpty = 6,
+  kVFull = 8,
+  kVEmpty = 10,
+  kSFull = 12,  // [2] per slot
+  kPFull = 14,
+  kODone = 16,
+  kOFree = 18,
+  kNumFwdBars = 20
+};
 
 template <int D>
 struct FwdSmem {
   static constexpr int kTileBytes = 128 * D * 2;
-  static constexpr int kQ = 0, kK = kTileBytes, kV = 2 * kTileBytes, kBars = 3 * kTileBytes;
-  static constexpr int kTotal = kBars + 64 + 1024;  // + slack to align the base to 1024 B
+  static constexpr int kQ = 0, kK = 2 * kTileBytes, kV = 4 * kTileBytes, kBars = 6 * kTileBytes;
+  static constexpr int kTotal = kBars + 256 + 1024;  // + slack to align the base to 1024 B
 };
 
+struct KvTile {
+  int start, len;
+  bool diag;
+};
+
+__device__ __forceinline__ KvTile kv_tile_of(const Tile& t, int j, int n0, int n1) {
+  KvTile k;
+  if (j < n0) {
+    k.start = t.kv0_start + j * kTile;
+    k.len = min(kTile, t.kv0_len - j * kTile);
+    k.diag = false;
+  } else if (j < n0 + n1) {
+    k.start = t.kv1_start + (j - n0) * kTile;
+    k.len = min(kTile, t.kv1_len - (j - n0) * kTile);
+    k.diag = false;
+  } else {
+    k.start = t.start;
+    k.len = t.len;
+    k.diag = true;
+  }
+  return k;
+}
+
+struct Unit {
+  Tile tile;
+  int h0, kvh, nslots, n0, n1, ntiles;
+};
+
+// Units are sorted longest first; CTA b takes unit b of round 0, the mirrored position of
+// round 1, and so on (boustrophedon), which evens out the per-CTA sums of a sorted list.
+__device__ __forceinline__ int unit_of_round(int round) {
+  const int g = gridDim.x, b = blockIdx.x;
+  return round * g + ((round & 1) ? (g - 1 - b) : b);
+}
+
+__device__ __forceinline__ bool get_unit(const FwdParams& prm, int u, int ntiles_total, Unit& un) {
+  const int r = prm.Hq / prm.Hkv, npairs = (r + 1) >> 1, per_tile = prm.Hkv * npairs;
+  const int ord = u / per_tile;
+  if (ord >= ntiles_total) return false;
+  const int rem = u - ord * per_tile;
+  un.kvh = rem / npairs;
+  const int pair = rem - un.kvh * npairs;
+  un.h0 = un.kvh * r + 2 * pair;
+  un.nslots = (2 * pair + 1 < r) ? 2 : 1;
+  un.tile = prm.tiles[prm.order[ord]];
+  un.n0 = (un.tile.kv0_len + kTile - 1) / kTile;
+  un.n1 = (un.tile.kv1_len + kTile - 1) / kTile;
+  un.ntiles = un.n0 + un.n1 + 1;
+  return true;
+}
+
 template <int D>
-__global__ void __launch_bounds__(kFwdThreads)
+__global__ void __launch_bounds__(kFwdThreads, 1)
 fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
            const __grid_constant__ CUtensorMap tm_v, FwdParams prm) {
   using L = FwdSmem<D>;
-  extern __shared__ uint8_t smem_raw[];
-  const int tid = threadIdx.x, warp = tid >> 5;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if (prm.header[0] != kStatusOk) return;
-  const int ord = blockIdx.x / prm.Hq, h = blockIdx.x % prm.Hq;
-  if (ord >= prm.header[2]) return;
-  const Tile tile = prm.tiles[prm.order[ord]];
-  const int kvh = h / (prm.Hq / prm.Hkv);
+  const int ntiles_total = prm.header[2];
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t sQ = base + L::kQ, sK = base + L::kK, sV = base + L::kV;
-  const uint32_t bar_q = base + L::kBars, bar_kv = bar_q + 8, bar_s = bar_q + 16,
-                 bar_o = bar_q + 24, tmem_slot = bar_q + 32;
   uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kBars + 40);
-  volatile uint32_t* tmem_slot_p = reinterpret_cast<volatile uint32_t*>(gbase + L::kBars + 32);
+  const uint32_t sQ = base + L::kQ, sK = base + L::kK, sV = base + L::kV;
+  const uint32_t bars = base + L::kBars;
+  auto bar = [&](int i) { return bars + 8u * uint32_t(i); };
+  const uint32_t tmem_slot = bars + 8 * kNumFwdBars;
+  volatile uint32_t* tmem_slot_p = reinterpret_cast<volatile uint32_t*>(gbase + L::kBars + 8 * kNumFwdBars);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kBars + 8 * kNumFwdBars + 8);
 
   if (tid == 0) {
-    mbar_init(bar_q, 1);
-    mbar_init(bar_kv, 1);
-    mbar_init(bar_s, 1);
-    mbar_init(bar_o, 1);
+    for (int i = 0; i < kNumFwdBars; ++i) {
+      const bool wg_count = (i >= kPFull && i < kPFull + 2) || (i >= kOFree && i < kOFree + 2);
+      mbar_init(bar(i), wg_count ? 128 : 1);
+    }
     *abort_flag = 0;
     fence_mbar_init();
     tma_prefetch_desc(&tm_q);
@@ -73,138 +146,211 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot_p;
-  const uint32_t lane_base = tmem + (uint32_t(warp * 32) << 16);
-  const uint32_t tS = 0, tP = 0, tO = 128;
 
-  constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);
-  constexpr uint32_t idesc_o = make_idesc(128, D, 0, 1);
-
-  if (tid == 0) {
-    mbar_expect_tx(bar_q, L::kTileBytes);
-    for (int b = 0; b < D / 64; ++b) tma_load_3d(sQ + b * kBoxBytes, &tm_q, b * 64, h, tile.start, bar_q);
-  }
-
-  const int n0 = (tile.kv0_len + kTile - 1) / kTile, n1 = (tile.kv1_len + kTile - 1) / kTile;
-  const int ntiles = n0 + n1 + 1;
-  float m_run = -INFINITY, l_run = 0.f;
-  const int row = tid;
-
-  for (int j = 0; j < ntiles; ++j) {
-    int k_start, k_len;
-    const bool diag = (j == ntiles - 1);
-    if (j < n0) {
-      k_start = tile.kv0_start + j * kTile;
-      k_len = min(kTile, tile.kv0_len - j * kTile);
-    } else if (j < n0 + n1) {
-      k_start = tile.kv1_start + (j - n0) * kTile;
-      k_len = min(kTile, tile.kv1_len - (j - n0) * kTile);
-    } else {
-      k_start = tile.start;
-      k_len = tile.len;
-    }
-    const uint32_t par = j & 1;
-
-    if (tid == 0) {
-      mbar_expect_tx(bar_kv, 2 * L::kTileBytes);
-      for (int b = 0; b < D / 64; ++b) {
-        tma_load_3d(sK + b * kBoxBytes, &tm_k, b * 64, kvh, k_start, bar_kv);
-        tma_load_3d(sV + b * kBoxBytes, &tm_v, b * 64, kvh, k_start, bar_kv);
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t kc = 0, vc = 0, qc[2] = {0, 0};
+      Unit un;
+      for (int rnd = 0; get_unit(prm, unit_of_round(rnd), ntiles_total, un); ++rnd) {
+        for (int s = 0; s < un.nslots; ++s) {
+          wait_bar(bar(kQEmpty + s), (qc[s] & 1) ^ 1, abort_flag, prm.header, 20 + s);
+          mbar_expect_tx(bar(kQFull + s), L::kTileBytes);
+          for (int b = 0; b < D / 64; ++b)
+            tma_load_3d(sQ + s * L::kTileBytes + b * kBoxBytes, &tm_q, b * 64, un.h0 + s,
+                        un.tile.start, bar(kQFull + s));
+          ++qc[s];
+        }
+        for (int j = 0; j < un.ntiles; ++j) {
+          const KvTile kt = kv_tile_of(un.tile, j, un.n0, un.n1);
+          uint32_t st = kc & 1;
+          wait_bar(bar(kKEmpty + st), ((kc >> 1) & 1) ^ 1, abort_flag, prm.header, 22);
+          mbar_expect_tx(bar(kKFull + st), L::kTileBytes);
+          for (int b = 0; b < D / 64; ++b)
+            tma_load_3d(sK + st * L::kTileBytes + b * kBoxBytes, &tm_k, b * 64, un.kvh, kt.start,
+                        bar(kKFull + st));
+          ++kc;
+          st = vc & 1;
+          wait_bar(bar(kVEmpty + st), ((vc >> 1) & 1) ^ 1, abort_flag, prm.header, 23);
+          mbar_expect_tx(bar(kVFull + st), L::kTileBytes);
+          for (int b = 0; b < D / 64; ++b)
+            tma_load_3d(sV + st * L::kTileBytes + b * kBoxBytes, &tm_v, b * 64, un.kvh, kt.start,
+                        bar(kVFull + st));
+          ++vc;
+        }
       }
-      if (j == 0) wait_bar(bar_q, 0, abort_flag, prm.header, 1);
-      wait_bar(bar_kv, par, abort_flag, prm.header, 2);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t kc = 0, vc = 0, tc[2] = {0, 0}, uc[2] = {0, 0};
+      constexpr uint32_t idesc_o = make_idesc(128, D, 0, 1);
+      Unit un;
+      auto issue_qk = [&](int s, uint32_t kstage, int k_len) {
+        const uint32_t idesc_s = make_idesc(128, ((k_len + 15) >> 4) << 4, 0, 0);
+        const uint32_t q = sQ + s * L::kTileBytes, k = sK + kstage * L::kTileBytes;
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk)
+          mma_ss(tmem + s * 128, kmajor_desc(q, kk), kmajor_desc(k, kk), idesc_s, kk > 0);
+        mma_commit(bar(kSFull + s));
+      };
+      for (int rnd = 0; get_unit(prm, unit_of_round(rnd), ntiles_total, un); ++rnd) {
+        for (int s = 0; s < un.nslots; ++s)
+          wait_bar(bar(kQFull + s), uc[s] & 1, abort_flag, prm.header, 30 + s);
+        KvTile kt = kv_tile_of(un.tile, 0, un.n0, un.n1);
+        wait_bar(bar(kKFull + (kc & 1)), (kc >> 1) & 1, abort_flag, prm.header, 32);
+        tc_fence_after();
+        for (int s = 0; s < un.nslots; ++s) {
+          issue_qk(s, kc & 1, kt.len);
+          if (un.ntiles == 1) mma_commit(bar(kQEmpty + s));
+        }
+        mma_commit(bar(kKEmpty + (kc & 1)));
+        ++kc;
+        for (int j = 0; j < un.ntiles; ++j) {
+          const bool has_next = j + 1 < un.ntiles;
+          const int cur_len = kt.len;
+          KvTile nx = kt;
+          if (has_next) nx = kv_tile_of(un.tile, j + 1, un.n0, un.n1);
+          wait_bar(bar(kVFull + (vc & 1)), (vc >> 1) & 1, abort_flag, prm.header, 33);
+          if (has_next)
+            wait_bar(bar(kKFull + (kc & 1)), (kc >> 1) & 1, abort_flag, prm.header, 34);
+          const uint32_t vbase = sV + (vc & 1) * L::kTileBytes;
+          for (int s = 0; s < un.nslots; ++s) {
+            wait_bar(bar(kPFull + s), tc[s] & 1, abort_flag, prm.header, 35 + s);
+            if (j == 0) wait_bar(bar(kOFree + s), (uc[s] & 1) ^ 1, abort_flag, prm.header, 37 + s);
+            tc_fence_after();
+            const int ksteps = (cur_len + 15) >> 4;
+            for (int kk = 0; kk < ksteps; ++kk)
+              mma_ts(tmem + 256 + s * 128, tmem + s * 128 + kk * 8, mnmajor_desc(vbase, kk), idesc_o,
+                     (j > 0) || (kk > 0));
+            mma_commit(bar(kODone + s));
+            ++tc[s];
+            if (has_next) {
+              issue_qk(s, kc & 1, nx.len);
+              if (j + 2 == un.ntiles) mma_commit(bar(kQEmpty + s));
+            }
+          }
+          mma_commit(bar(kVEmpty + (vc & 1)));
+          ++vc;
+          if (has_next) {
+            mma_commit(bar(kKEmpty + (kc & 1)));
+            ++kc;
+          }
+          kt = nx;
+        }
+        for (int s = 0; s < un.nslots; ++s) ++uc[s];
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ softmax warpgroups
+    const int s = (warp - 2) >> 2;
+    const int row = 32 * (warp & 3) + lane;
+    const uint32_t lane_base = tmem + (uint32_t(32 * (warp & 3)) << 16);
+    const uint32_t tS = lane_base + s * 128, tO = lane_base + 256 + s * 128;
+    uint32_t tcS = 0;
+    Unit un;
+    for (int rnd = 0; get_unit(prm, unit_of_round(rnd), ntiles_total, un); ++rnd) {
+      if (s >= un.nslots) continue;
+      float m_used = -INFINITY, l_run = 0.f;
+      for (int j = 0; j < un.ntiles; ++j) {
+        const KvTile kt = kv_tile_of(un.tile, j, un.n0, un.n1);
+        wait_bar(bar(kSFull + s), tcS & 1, abort_flag, prm.header, 40 + s);
+        tc_fence_after();
+        uint32_t v[128];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[c * 32]));
+        tmem_wait_ld();
+        const bool full = !kt.diag && kt.len == kTile;
+        const int col_lim = kt.diag ? min(kt.len, row + 1) : kt.len;
+        float mx = -INFINITY;
+        if (full) {
+#pragma unroll
+          for (int i = 0; i < 128; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
+        } else {
+#pragma unroll
+          for (int i = 0; i < 128; ++i)
+            mx = fmaxf(mx, i < col_lim ? __uint_as_float(v[i]) : -INFINITY);
+        }
+        mx *= prm.scale_log2;
+        if (j == 0) {
+          m_used = mx;
+        } else {
+          const float m_new = fmaxf(m_used, mx);
+          const bool need = (m_new - m_used) > kRescaleThreshold;
+          if (__any_sync(0xffffffffu, need)) {
+            const float alpha = ex2(m_used - m_new);
+            wait_bar(bar(kODone + s), (tcS - 1) & 1, abort_flag, prm.header, 42 + s);
+            tc_fence_after();
+#pragma unroll 1
+            for (int c = 0; c < D / 32; ++c) {
+              uint32_t w[32];
+              tmem_ld32(tO + c * 32, w);
+              tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) w[i] = __float_as_uint(__uint_as_float(w[i]) * alpha);
+              tmem_st32(tO + c * 32, w);
+            }
+            l_run *= alpha;
+            m_used = m_new;
+          }
+        }
+        float rs = 0.f;
+        const float neg_m = -m_used;
+        if (full) {
+#pragma unroll
+          for (int i = 0; i < 64; ++i) {
+            const float p0 = ex2(fmaf(__uint_as_float(v[2 * i]), prm.scale_log2, neg_m));
+            const float p1 = ex2(fmaf(__uint_as_float(v[2 * i + 1]), prm.scale_log2, neg_m));
+            rs += p0 + p1;
+            v[i] = pack_bf16(p0, p1);
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 64; ++i) {
+            float p0 = ex2(fmaf(__uint_as_float(v[2 * i]), prm.scale_log2, neg_m));
+            float p1 = ex2(fmaf(__uint_as_float(v[2 * i + 1]), prm.scale_log2, neg_m));
+            p0 = (2 * i < col_lim) ? p0 : 0.f;
+            p1 = (2 * i + 1 < col_lim) ? p1 : 0.f;
+            rs += p0 + p1;
+            v[i] = pack_bf16(p0, p1);
+          }
+        }
+        l_run += rs;
+        tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+        tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(kPFull + s));
+        ++tcS;
+      }
+      // ---- epilogue: O / l -> bf16 registers, release the accumulator, then store
+      wait_bar(bar(kODone + s), (tcS - 1) & 1, abort_flag, prm.header, 44 + s);
       tc_fence_after();
+      const float inv_l = 1.f / l_run;
+      uint32_t ob[D / 2];
 #pragma unroll
-      for (int k = 0; k < D / 16; ++k)
-        mma_ss(tmem + tS, kmajor_desc(sQ, k), kmajor_desc(sK, k), idesc_s, k > 0);
-      mma_commit(bar_s);
-    }
-    wait_bar(bar_s, par, abort_flag, prm.header, 3);
-    tc_fence_after();
-
-    // ---- online softmax on this thread's row (base-2 exponentials)
-    uint32_t v[32];
-    float mx = m_run;
-    const int col_lim = diag ? min(k_len, row + 1) : k_len;  // columns [0, col_lim) are visible
-#pragma unroll 1
-    for (int c = 0; c < 4; ++c) {
-      tmem_ld32(lane_base + tS + c * 32, v);
-      tmem_wait_ld();
-#pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        float s = __uint_as_float(v[i]) * prm.scale_log2;
-        if (c * 32 + i < col_lim) mx = fmaxf(mx, s);
-      }
-    }
-    const float alpha = ex2(m_run - mx);
-    float rs = 0.f;
-#pragma unroll 1
-    for (int c = 0; c < 4; ++c) {
-      tmem_ld32(lane_base + tS + c * 32, v);
-      tmem_wait_ld();
-      uint32_t pk[16];
-#pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        int c0 = c * 32 + 2 * i;
-        float p0 = ex2(__uint_as_float(v[2 * i]) * prm.scale_log2 - mx);
-        float p1 = ex2(__uint_as_float(v[2 * i + 1]) * prm.scale_log2 - mx);
-        p0 = (c0 < col_lim) ? p0 : 0.f;
-        p1 = (c0 + 1 < col_lim) ? p1 : 0.f;
-        rs += p0 + p1;
-        pk[i] = pack_bf16(p0, p1);
-      }
-      tmem_st16(lane_base + tP + c * 16, pk);
-    }
-    l_run = l_run * alpha + rs;
-    m_run = mx;
-    if (j > 0) {
-#pragma unroll 1
       for (int c = 0; c < D / 32; ++c) {
-        tmem_ld32(lane_base + tO + c * 32, v);
+        uint32_t w[32];
+        tmem_ld32(tO + c * 32, w);
         tmem_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-        tmem_st32(lane_base + tO + c * 32, v);
+        for (int i = 0; i < 16; ++i)
+          ob[c * 16 + i] = pack_bf16(__uint_as_float(w[2 * i]) * inv_l, __uint_as_float(w[2 * i + 1]) * inv_l);
       }
-    }
-    tmem_wait_st();
-    tc_fence_before();
-    __syncthreads();
-
-    if (tid == 0) {
-      tc_fence_after();
-      const int ksteps = (k_len + 15) / 16;
-      for (int k = 0; k < ksteps; ++k)
-        mma_ts(tmem + tO, tmem + tP + k * 8, mnmajor_desc(sV, k), idesc_o, (j > 0) || (k > 0));
-      mma_commit(bar_o);
-    }
-    wait_bar(bar_o, par, abort_flag, prm.header, 4);
-    tc_fence_after();
-  }
-
-  // ---- epilogue: normalise, round to bf16, store this thread's row; LSE in natural log
-  const float inv_l = 1.f / l_run;
-  if (row < tile.len) {
-    const size_t tok = size_t(tile.start) + row;
-    prm.lse[size_t(h) * prm.T + tok] = (m_run + log2f(l_run)) * 0.69314718055994531f;
-  }
-#pragma unroll 1
-  for (int c = 0; c < D / 32; ++c) {
-    uint32_t v[32];
-    tmem_ld32(lane_base + tO + c * 32, v);
-    tmem_wait_ld();
-    if (row < tile.len) {
-      uint4* dst = reinterpret_cast<uint4*>(prm.o + ((size_t(tile.start) + row) * prm.Hq + h) * D + c * 32);
+      tc_fence_before();
+      mbar_arrive(bar(kOFree + s));
+      if (row < un.tile.len) {
+        const int h = un.h0 + s;
+        const size_t tok = size_t(un.tile.start) + row;
+        prm.lse[size_t(h) * prm.T + tok] = (m_used + log2f(l_run)) * 0.69314718055994531f;
+        uint4* dst = reinterpret_cast<uint4*>(prm.o + (tok * prm.Hq + h) * D);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        uint4 w;
-        w.x = pack_bf16(__uint_as_float(v[8 * i + 0]) * inv_l, __uint_as_float(v[8 * i + 1]) * inv_l);
-        w.y = pack_bf16(__uint_as_float(v[8 * i + 2]) * inv_l, __uint_as_float(v[8 * i + 3]) * inv_l);
-        w.z = pack_bf16(__uint_as_float(v[8 * i + 4]) * inv_l, __uint_as_float(v[8 * i + 5]) * inv_l);
-        w.w = pack_bf16(__uint_as_float(v[8 * i + 6]) * inv_l, __uint_as_float(v[8 * i + 7]) * inv_l);
-        dst[i] = w;
+        for (int i = 0; i < D / 8; ++i)
+          dst[i] = make_uint4(ob[4 * i], ob[4 * i + 1], ob[4 * i + 2], ob[4 * i + 3]);
       }
     }
   }
+
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, kFwdTmemCols);
@@ -214,14 +360,22 @@ template <int D>
 cudaError_t launch_fwd_t(const pp_plan* plan, const CUtensorMap& tq, const CUtensorMap& tk,
                          const CUtensorMap& tv, const FwdParams& prm, cudaStream_t stream) {
   static bool configured = false;
+  static int num_sms = 0;
   auto kern = fwd_kernel<D>;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          FwdSmem<D>::kTotal);
     if (e != cudaSuccess) return e;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
     configured = true;
   }
-  dim3 grid(unsigned(plan->max_tiles) * unsigned(plan->prob.num_q_heads));
+  const pp_problem& pb = plan->prob;
+  const int r = pb.num_q_heads / pb.num_kv_heads;
+  const long long units = (long long)plan->max_tiles * pb.num_kv_heads * ((r + 1) / 2);
+  dim3 grid(unsigned(std::min<long long>(units, num_sms)));
   ProfileEvents& ev = profile_events();
   if (ev.on) cudaEventRecord(ev.fwd0, stream);
   kern<<<grid, kFwdThreads, FwdSmem<D>::kTotal, stream>>>(tq, tk, tv, prm);
