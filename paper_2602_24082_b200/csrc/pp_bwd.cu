@@ -76,49 +76,126 @@ bwd_finalize_kernel(const float4* __restrict__ acc, uint2* __restrict__ dq, size
 }
 
 // ---------------------------------------------------------------- main
-constexpr int kBwdThreads = 128;
-constexpr uint32_t kBwdTmemCols = 512;  // S^T/P^T [0,128) | dP^T/dQ [128,256) | dV [256,..) | dK [384,..)
+// Persistent, warp-specialised CTA (one per SM), 448 threads:
+//   warp 0       producer: K, V once per unit; per query tile Q and dO by TMA (two-stage rings)
+//                and the tile's LSE*log2(e) / Delta into shared memory
+//   warp 1       MMA issuer (one thread)
+//   warps 2-5    compute warpgroup 0: thread = key row, query columns 0..63 of the tile
+//   warps 6-9    compute warpgroup 1: query columns 64..127
+//   warps 10-13  dQ warpgroup: thread = query row, drains dQ tiles into the fp32 accumulator
+// Tensor-memory map (columns): [0,128) S^T, overwritten by P^T (bf16: columns [0,32) and
+// [64,96), each warpgroup inside the columns it has read itself); [128,256) dP^T, then the
+// dQ tile; [256,256+D) dV; [384,384+D) dK.
+// MMA order per query tile i:  dP(i)  dV(i)  S(i+1)  dQ(i)  dK(i).  The exponentials of tile
+// i+1 run under dQ(i), dK(i), dP(i+1); dS(i) is computed under dV(i), S(i+1); the dQ tile is
+// drained under dK(i), so the dP/dQ columns are free again when dP(i+1) is issued.
+constexpr int kBwdThreads = 448;
+constexpr uint32_t kBwdTmemCols = 512;
+
+enum BwdBar : int {
+  kKvFull = 0,
+  kKvEmpty,
+  kQFullB,       // [2]   33 arrivals: TMA transaction + 32 producer lanes (LSE / Delta)
+  kQEmptyB = 4,  // [2]
+  kDoFull = 6,   // [2]
+  kDoEmpty = 8,  // [2]
+  kSFullB = 10,
+  kPReady,       // 256
+  kDpFull,
+  kDsReady,      // 256
+  kDqFull,
+  kDqDrained,    // 128
+  kDkvFull,
+  kDkvFree,      // 256
+  kNumBwdBars
+};
 
 template <int D>
 struct BwdSmem {
   static constexpr int kTileBytes = 128 * D * 2;
-  static constexpr int kK = 0, kV = kTileBytes, kQ = 2 * kTileBytes, kdO = 3 * kTileBytes,
-                       kdS = 4 * kTileBytes, kLse = kdS + 128 * 128 * 2, kDelta = kLse + 512,
-                       kBars = kDelta + 512;
-  static constexpr int kTotal = kBars + 64 + 1024;
+  static constexpr int kK = 0, kV = kTileBytes, kQ = 2 * kTileBytes, kdO = 4 * kTileBytes,
+                       kdS = 6 * kTileBytes, kStats = kdS + 128 * 128 * 2,
+                       kBars = kStats + 2 * 256 * 4;
+  static constexpr int kUsed = kBars + 8 * kNumBwdBars + 16;
+  // The declared 1024-byte alignment of the dynamic shared memory leaves no slack to spend at
+  // D = 128 (227 KB limit); the kernel checks the base and reports if it is not aligned.
+  static constexpr int kTotal = kUsed + (kUsed + 1024 <= 232448 ? 1024 : 0);
 };
 
+struct BwdUnit {
+  Tile tile;
+  int kvh, nq, n_it;
+};
+
+__device__ __forceinline__ int bwd_unit_of_round(int round) {
+  const int g = gridDim.x, b = blockIdx.x;
+  return round * g + ((round & 1) ? (g - 1 - b) : b);
+}
+
+__device__ __forceinline__ bool get_bwd_unit(const BwdParams& prm, int u, int ntiles_total,
+                                             BwdUnit& un) {
+  const int ord = u / prm.Hkv;
+  if (ord >= ntiles_total) return false;
+  un.kvh = u - ord * prm.Hkv;
+  un.tile = prm.tiles[prm.order[ord]];
+  const int full_len = un.tile.vis_end - (un.tile.start + un.tile.len);
+  un.nq = 1 + (full_len + kTile - 1) / kTile;
+  un.n_it = un.nq * (prm.Hq / prm.Hkv);
+  return true;
+}
+
+struct QTile {
+  int h, start, len;
+  bool diag;
+};
+
+__device__ __forceinline__ QTile q_tile_of(const BwdParams& prm, const BwdUnit& un, int it) {
+  QTile q;
+  const int hh = it / un.nq, qt = it - hh * un.nq;
+  q.h = un.kvh * (prm.Hq / prm.Hkv) + hh;
+  q.diag = (qt == 0);
+  q.start = q.diag ? un.tile.start : un.tile.start + un.tile.len + (qt - 1) * kTile;
+  q.len = q.diag ? un.tile.len : min(kTile, un.tile.vis_end - q.start);
+  return q;
+}
+
 template <int D>
-__global__ void __launch_bounds__(kBwdThreads)
+__global__ void __launch_bounds__(kBwdThreads, 1)
 bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
            const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
            BwdParams prm) {
   using L = BwdSmem<D>;
-  extern __shared__ uint8_t smem_raw[];
-  const int tid = threadIdx.x, warp = tid >> 5;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if (prm.header[0] != kStatusOk) return;
-  const int ord = blockIdx.x / prm.Hkv, kvh = blockIdx.x % prm.Hkv;
-  if (ord >= prm.header[2]) return;
-  const Tile tile = prm.tiles[prm.order[ord]];
-  const int r = prm.Hq / prm.Hkv;
+  const int ntiles_total = prm.header[2];
 
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  if (base - raw + L::kUsed > L::kTotal) {  // cannot happen with an aligned base
+    if (tid == 0 && atomicCAS(&prm.header[0], kStatusOk, kStatusWaitExpired) == kStatusOk)
+      prm.header[1] = 99;
+    return;
+  }
+  uint8_t* gbase = smem_raw + (base - raw);
   const uint32_t sK = base + L::kK, sV = base + L::kV, sQ = base + L::kQ, sdO = base + L::kdO,
                  sdS = base + L::kdS;
-  float* sLse = reinterpret_cast<float*>(gbase + L::kLse);
-  float* sDelta = reinterpret_cast<float*>(gbase + L::kDelta);
-  const uint32_t bar_kv = base + L::kBars, bar_ld = bar_kv + 8, bar_s = bar_kv + 16,
-                 bar_d = bar_kv + 24, tmem_slot = bar_kv + 32;
-  volatile uint32_t* tmem_slot_p = reinterpret_cast<volatile uint32_t*>(gbase + L::kBars + 32);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kBars + 40);
+  float* stats = reinterpret_cast<float*>(gbase + L::kStats);  // [stage][lse2 128 | delta 128]
+  const uint32_t bars = base + L::kBars;
+  auto bar = [&](int i) { return bars + 8u * uint32_t(i); };
+  const uint32_t tmem_slot = bars + 8 * kNumBwdBars;
+  volatile uint32_t* tmem_slot_p = reinterpret_cast<volatile uint32_t*>(gbase + L::kBars + 8 * kNumBwdBars);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kBars + 8 * kNumBwdBars + 8);
 
   if (tid == 0) {
-    mbar_init(bar_kv, 1);
-    mbar_init(bar_ld, 1);
-    mbar_init(bar_s, 1);
-    mbar_init(bar_d, 1);
+    for (int i = 0; i < kNumBwdBars; ++i) {
+      uint32_t cnt = 1;
+      if (i == kQFullB || i == kQFullB + 1) cnt = 33;
+      if (i == kPReady || i == kDsReady || i == kDkvFree) cnt = 256;
+      if (i == kDqDrained) cnt = 128;
+      mbar_init(bar(i), cnt);
+    }
     *abort_flag = 0;
     fence_mbar_init();
     tma_prefetch_desc(&tm_q);
@@ -134,164 +211,259 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot_p;
-  const uint32_t lane_base = tmem + (uint32_t(warp * 32) << 16);
-  constexpr uint32_t tS = 0, tP = 0, tdP = 128, tdQ = 128, tdV = 256, tdK = 384;
+  constexpr uint32_t tS = 0, tdP = 128, tdV = 256, tdK = 384;
 
-  constexpr uint32_t idesc_st = make_idesc(128, 128, 0, 0);  // S^T, dP^T : K-major x K-major
-  constexpr uint32_t idesc_kv = make_idesc(128, D, 0, 1);    // dV, dK    : K-major A, MN-major B
-  constexpr uint32_t idesc_dq = make_idesc(128, D, 1, 1);    // dQ        : MN-major A and B
-
-  const int k_start = tile.start, k_len = tile.len;
-  if (tid == 0) {
-    mbar_expect_tx(bar_kv, 2 * L::kTileBytes);
-    for (int b = 0; b < D / 64; ++b) {
-      tma_load_3d(sK + b * kBoxBytes, &tm_k, b * 64, kvh, k_start, bar_kv);
-      tma_load_3d(sV + b * kBoxBytes, &tm_v, b * 64, kvh, k_start, bar_kv);
-    }
-  }
-
-  const int full_len = tile.vis_end - (k_start + k_len);
-  const int nq = 1 + (full_len + kTile - 1) / kTile;
-  const int lane = tid;  // TMEM lane = key row (S^T, dP^T, dK, dV) or query row (dQ)
-
-  int it = 0;
-  for (int hh = 0; hh < r; ++hh) {
-    const int h = kvh * r + hh;
-    for (int qt = 0; qt < nq; ++qt, ++it) {
-      const bool diag = (qt == 0);
-      const int q_start = diag ? k_start : k_start + k_len + (qt - 1) * kTile;
-      const int q_len = diag ? k_len : min(kTile, tile.vis_end - q_start);
-      const uint32_t par = it & 1;
-
-      if (tid == 0) {
-        mbar_expect_tx(bar_ld, 2 * L::kTileBytes);
+  if (warp == 0) {
+    // ------------------------------------------------------------ producer
+    uint32_t qc = 0, ucnt = 0;
+    BwdUnit un;
+    for (int rnd = 0; get_bwd_unit(prm, bwd_unit_of_round(rnd), ntiles_total, un); ++rnd, ++ucnt) {
+      if (lane == 0) {
+        wait_bar(bar(kKvEmpty), (ucnt & 1) ^ 1, abort_flag, prm.header, 50);
+        mbar_expect_tx(bar(kKvFull), 2 * L::kTileBytes);
         for (int b = 0; b < D / 64; ++b) {
-          tma_load_3d(sQ + b * kBoxBytes, &tm_q, b * 64, h, q_start, bar_ld);
-          tma_load_3d(sdO + b * kBoxBytes, &tm_do, b * 64, h, q_start, bar_ld);
+          tma_load_3d(sK + b * kBoxBytes, &tm_k, b * 64, un.kvh, un.tile.start, bar(kKvFull));
+          tma_load_3d(sV + b * kBoxBytes, &tm_v, b * 64, un.kvh, un.tile.start, bar(kKvFull));
         }
       }
-      // per-query statistics of this tile; +inf LSE switches off queries past the tile's end
-      sLse[tid] = tid < q_len ? prm.lse2[size_t(h) * prm.T + q_start + tid] : INFINITY;
-      sDelta[tid] = tid < q_len ? prm.delta[size_t(h) * prm.T + q_start + tid] : 0.f;
-
-      if (tid == 0) {
-        if (it == 0) wait_bar(bar_kv, 0, abort_flag, prm.header, 11);
-        wait_bar(bar_ld, par, abort_flag, prm.header, 12);
-        tc_fence_after();
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k)
-          mma_ss(tmem + tS, kmajor_desc(sK, k), kmajor_desc(sQ, k), idesc_st, k > 0);
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k)
-          mma_ss(tmem + tdP, kmajor_desc(sV, k), kmajor_desc(sdO, k), idesc_st, k > 0);
-        mma_commit(bar_s);
-      }
-      __syncthreads();  // sLse / sDelta visible
-      wait_bar(bar_s, par, abort_flag, prm.header, 13);
-      tc_fence_after();
-
-      const bool row_ok = lane < k_len;
-#pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        uint32_t v[32];
-        float p[32];
-        tmem_ld32(lane_base + tS + c * 32, v);
-        tmem_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const int col = c * 32 + i;
-          float e = ex2(__uint_as_float(v[i]) * prm.scale_log2 - sLse[col]);
-          const bool vis = row_ok && (!diag || col >= lane);
-          p[i] = vis ? e : 0.f;
+      for (int it = 0; it < un.n_it; ++it, ++qc) {
+        const QTile qt = q_tile_of(prm, un, it);
+        const uint32_t st = qc & 1, par = ((qc >> 1) & 1) ^ 1;
+        wait_bar(bar(kQEmptyB + st), par, abort_flag, prm.header, 51);
+        if (lane == 0) {
+          mbar_expect_tx(bar(kQFullB + st), L::kTileBytes);
+          for (int b = 0; b < D / 64; ++b)
+            tma_load_3d(sQ + st * L::kTileBytes + b * kBoxBytes, &tm_q, b * 64, qt.h, qt.start,
+                        bar(kQFullB + st));
         }
-        uint32_t pk[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(p[2 * i], p[2 * i + 1]);
-        tmem_st16(lane_base + tP + c * 16, pk);
-
-        tmem_ld32(lane_base + tdP + c * 32, v);
-        tmem_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const int col = c * 32 + 2 * i;
-          float d0 = p[2 * i] * (__uint_as_float(v[2 * i]) - sDelta[col]);
-          float d1 = p[2 * i + 1] * (__uint_as_float(v[2 * i + 1]) - sDelta[col + 1]);
-          pk[i] = pack_bf16(d0, d1);
-        }
-        // dS^T row `lane`, columns [32c, 32c+32): box c/2, 16-byte chunks (c%2)*4 .. +3, swizzled
-        const uint32_t row_addr = sdS + (c >> 1) * kBoxBytes + lane * 128;
+        // per-query statistics; +inf LSE and zero Delta switch off columns past the tile's end
+        float* sl = stats + st * 256;
+        const size_t row0 = size_t(qt.h) * prm.T + qt.start;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const uint32_t chunk = uint32_t((c & 1) * 4 + i) ^ uint32_t(lane & 7);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + chunk * 16),
-                       "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]), "r"(pk[4 * i + 3])
-                       : "memory");
+          const int c = lane + 32 * i;
+          sl[c] = c < qt.len ? prm.lse2[row0 + c] : INFINITY;
+          sl[128 + c] = c < qt.len ? prm.delta[row0 + c] : 0.f;
+        }
+        mbar_arrive(bar(kQFullB + st));
+        if (lane == 0) {
+          wait_bar(bar(kDoEmpty + st), par, abort_flag, prm.header, 52);
+          mbar_expect_tx(bar(kDoFull + st), L::kTileBytes);
+          for (int b = 0; b < D / 64; ++b)
+            tma_load_3d(sdO + st * L::kTileBytes + b * kBoxBytes, &tm_do, b * 64, qt.h, qt.start,
+                        bar(kDoFull + st));
         }
       }
-      tmem_wait_st();
-      fence_proxy_async_smem();
-      tc_fence_before();
-      __syncthreads();
-
-      if (tid == 0) {
-        tc_fence_after();
-        const int qsteps = (q_len + 15) / 16, ksteps = (k_len + 15) / 16;
-        for (int k = 0; k < qsteps; ++k)
-          mma_ts(tmem + tdV, tmem + tP + k * 8, mnmajor_desc(sdO, k), idesc_kv, (it > 0) || (k > 0));
-        for (int k = 0; k < qsteps; ++k)
-          mma_ss(tmem + tdK, kmajor_desc(sdS, k), mnmajor_desc(sQ, k), idesc_kv, (it > 0) || (k > 0));
-        for (int k = 0; k < ksteps; ++k)
-          mma_ss(tmem + tdQ, mnmajor_desc(sdS, k), mnmajor_desc(sK, k), idesc_dq, k > 0);
-        mma_commit(bar_d);
-      }
-      wait_bar(bar_d, par, abort_flag, prm.header, 14);
-      tc_fence_after();
-
-      // dQ tile: lane = query row; add into the fp32 accumulator
-#pragma unroll 1
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t v[32];
-        tmem_ld32(lane_base + tdQ + c * 32, v);
-        tmem_wait_ld();
-        if (lane < q_len) {
-          float* dst = prm.dq_acc + ((size_t(q_start) + lane) * prm.Hq + h) * D + c * 32;
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t gc = 0, ucnt = 0;
+      constexpr uint32_t idesc_kv = make_idesc(128, D, 0, 1);  // dV, dK : K-major A, MN-major B
+      constexpr uint32_t idesc_dq = make_idesc(128, D, 1, 1);  // dQ     : MN-major A and B
+      BwdUnit un;
+      auto issue_s = [&](uint32_t st, int q_len) {
+        const uint32_t idesc = make_idesc(128, ((q_len + 15) >> 4) << 4, 0, 0);
+        const uint32_t q = sQ + st * L::kTileBytes;
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
+        for (int k = 0; k < D / 16; ++k)
+          mma_ss(tmem + tS, kmajor_desc(sK, k), kmajor_desc(q, k), idesc, k > 0);
+        mma_commit(bar(kSFullB));
+      };
+      for (int rnd = 0; get_bwd_unit(prm, bwd_unit_of_round(rnd), ntiles_total, un); ++rnd, ++ucnt) {
+        const int ksteps = (un.tile.len + 15) >> 4;
+        wait_bar(bar(kKvFull), ucnt & 1, abort_flag, prm.header, 60);
+        QTile qt = q_tile_of(prm, un, 0);
+        wait_bar(bar(kQFullB + (gc & 1)), (gc >> 1) & 1, abort_flag, prm.header, 61);
+        tc_fence_after();
+        issue_s(gc & 1, qt.len);
+        for (int it = 0; it < un.n_it; ++it) {
+          const uint32_t g = gc + it, st = g & 1, spar = (g >> 1) & 1, par = g & 1;
+          const int qsteps = (qt.len + 15) >> 4;
+          const uint32_t q = sQ + st * L::kTileBytes, d_o = sdO + st * L::kTileBytes;
+          // dP^T(it) = V dO^T
+          wait_bar(bar(kDoFull + st), spar, abort_flag, prm.header, 62);
+          if (g > 0) wait_bar(bar(kDqDrained), (g - 1) & 1, abort_flag, prm.header, 63);
+          tc_fence_after();
+          {
+            const uint32_t idesc = make_idesc(128, qsteps << 4, 0, 0);
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k)
+              mma_ss(tmem + tdP, kmajor_desc(sV, k), kmajor_desc(d_o, k), idesc, k > 0);
+            mma_commit(bar(kDpFull));
+          }
+          // dV += P^T dO
+          wait_bar(bar(kPReady), par, abort_flag, prm.header, 64);
+          if (it == 0) wait_bar(bar(kDkvFree), (ucnt & 1) ^ 1, abort_flag, prm.header, 65);
+          tc_fence_after();
+          for (int k = 0; k < qsteps; ++k)
+            mma_ts(tmem + tdV, tmem + tS + (k < 4 ? k * 8 : 64 + (k - 4) * 8), mnmajor_desc(d_o, k),
+                   idesc_kv, (it > 0) || (k > 0));
+          mma_commit(bar(kDoEmpty + st));
+          // S^T(it+1) = K Q^T
+          QTile nx = qt;
+          if (it + 1 < un.n_it) {
+            nx = q_tile_of(prm, un, it + 1);
+            const uint32_t g1 = g + 1;
+            wait_bar(bar(kQFullB + (g1 & 1)), (g1 >> 1) & 1, abort_flag, prm.header, 66);
+            tc_fence_after();
+            issue_s(g1 & 1, nx.len);
+          }
+          // dQ(it) = dS K, then dK += dS^T Q
+          wait_bar(bar(kDsReady), par, abort_flag, prm.header, 67);
+          tc_fence_after();
+          for (int k = 0; k < ksteps; ++k)
+            mma_ss(tmem + tdP, mnmajor_desc(sdS, k), mnmajor_desc(sK, k), idesc_dq, k > 0);
+          mma_commit(bar(kDqFull));
+          for (int k = 0; k < qsteps; ++k)
+            mma_ss(tmem + tdK, kmajor_desc(sdS, k), mnmajor_desc(q, k), idesc_kv, (it > 0) || (k > 0));
+          mma_commit(bar(kQEmptyB + st));
+          qt = nx;
+        }
+        mma_commit(bar(kDkvFull));
+        mma_commit(bar(kKvEmpty));
+        gc += un.n_it;
+      }
+    }
+  } else if (warp < 10) {
+    // ------------------------------------------------------------ compute warpgroups
+    const int wg = (warp - 2) >> 2;       // column half
+    const int row = 32 * (warp & 3) + lane;
+    const uint32_t lane_base = tmem + (uint32_t(32 * (warp & 3)) << 16);
+    const int cb = 64 * wg;
+    uint32_t gc = 0, ucnt = 0;
+    BwdUnit un;
+    for (int rnd = 0; get_bwd_unit(prm, bwd_unit_of_round(rnd), ntiles_total, un); ++rnd, ++ucnt) {
+      const bool row_ok = row < un.tile.len;
+      for (int it = 0; it < un.n_it; ++it) {
+        const QTile qt = q_tile_of(prm, un, it);
+        const uint32_t g = gc + it, st = g & 1, par = g & 1;
+        const float* sl = stats + st * 256 + cb;
+        const bool full = !qt.diag && qt.len == kTile && un.tile.len == kTile;
+        wait_bar(bar(kQFullB + st), (g >> 1) & 1, abort_flag, prm.header, 70);
+        wait_bar(bar(kSFullB), par, abort_flag, prm.header, 71);
+        tc_fence_after();
+        uint32_t v[64];
+        tmem_ld32(lane_base + tS + cb, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+        tmem_ld32(lane_base + tS + cb + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
+        tmem_wait_ld();
+        uint32_t pk[32];
+        if (full) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float p0 = ex2(fmaf(__uint_as_float(v[2 * i]), prm.scale_log2, -sl[2 * i]));
+            const float p1 = ex2(fmaf(__uint_as_float(v[2 * i + 1]), prm.scale_log2, -sl[2 * i + 1]));
+            pk[i] = pack_bf16(p0, p1);
+          }
+        } else {
+          // visible iff the key row exists, the query column exists, and (diagonal tile) the
+          // query is not before the key
+          const int lo = qt.diag ? row : 0;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int c0 = cb + 2 * i;
+            float p0 = ex2(fmaf(__uint_as_float(v[2 * i]), prm.scale_log2, -sl[2 * i]));
+            float p1 = ex2(fmaf(__uint_as_float(v[2 * i + 1]), prm.scale_log2, -sl[2 * i + 1]));
+            p0 = (row_ok && c0 >= lo && c0 < qt.len) ? p0 : 0.f;
+            p1 = (row_ok && c0 + 1 >= lo && c0 + 1 < qt.len) ? p1 : 0.f;
+            pk[i] = pack_bf16(p0, p1);
+          }
+        }
+        tmem_st32(lane_base + tS + cb, pk);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(kPReady));
+
+        wait_bar(bar(kDpFull), par, abort_flag, prm.header, 72);
+        tc_fence_after();
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          uint32_t d[32];
+          tmem_ld32(lane_base + tdP + cb + 32 * half, d);
+          tmem_wait_ld();
+          uint32_t ds[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const uint32_t pp = pk[16 * half + i];
+            const float p0 = __uint_as_float(pp << 16), p1 = __uint_as_float(pp & 0xffff0000u);
+            float d0 = p0 * (__uint_as_float(d[2 * i]) - sl[128 + 32 * half + 2 * i]);
+            float d1 = p1 * (__uint_as_float(d[2 * i + 1]) - sl[128 + 32 * half + 2 * i + 1]);
+            if (!full) {  // stale tensor-memory columns may hold anything
+              d0 = (pp & 0xffffu) ? d0 : 0.f;
+              d1 = (pp & 0xffff0000u) ? d1 : 0.f;
+            }
+            ds[i] = pack_bf16(d0, d1);
+          }
+          // dS^T row `row`, columns [cb + 32 half, +32): box wg, 16-byte chunks 4 half .. +3
+          const uint32_t row_addr = sdS + wg * kBoxBytes + row * 128;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint32_t chunk = uint32_t(half * 4 + i) ^ uint32_t(row & 7);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + chunk * 16),
+                         "r"(ds[4 * i]), "r"(ds[4 * i + 1]), "r"(ds[4 * i + 2]), "r"(ds[4 * i + 3])
+                         : "memory");
+          }
+        }
+        fence_proxy_async_smem();
+        mbar_arrive(bar(kDsReady));
+      }
+      gc += un.n_it;
+      // ---- unit epilogue: warpgroup 0 stores dV, warpgroup 1 stores scale * dK
+      wait_bar(bar(kDkvFull), ucnt & 1, abort_flag, prm.header, 73);
+      tc_fence_after();
+      const uint32_t tsrc = wg ? tdK : tdV;
+      const float f = wg ? prm.scale : 1.f;
+      uint32_t ob[D / 2];
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t w[32];
+        tmem_ld32(lane_base + tsrc + c * 32, w);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          ob[c * 16 + i] = pack_bf16(__uint_as_float(w[2 * i]) * f, __uint_as_float(w[2 * i + 1]) * f);
+      }
+      tc_fence_before();
+      mbar_arrive(bar(kDkvFree));
+      if (row_ok) {
+        __nv_bfloat16* out = wg ? prm.dk : prm.dv;
+        uint4* dst = reinterpret_cast<uint4*>(out + ((size_t(un.tile.start) + row) * prm.Hkv + un.kvh) * D);
+#pragma unroll
+        for (int i = 0; i < D / 8; ++i)
+          dst[i] = make_uint4(ob[4 * i], ob[4 * i + 1], ob[4 * i + 2], ob[4 * i + 3]);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ dQ warpgroup
+    const int row = 32 * (warp & 3) + lane;
+    const uint32_t lane_base = tmem + (uint32_t(32 * (warp & 3)) << 16);
+    uint32_t gc = 0;
+    BwdUnit un;
+    for (int rnd = 0; get_bwd_unit(prm, bwd_unit_of_round(rnd), ntiles_total, un); ++rnd) {
+      for (int it = 0; it < un.n_it; ++it) {
+        const QTile qt = q_tile_of(prm, un, it);
+        const uint32_t g = gc + it;
+        wait_bar(bar(kDqFull), g & 1, abort_flag, prm.header, 80);
+        tc_fence_after();
+        uint32_t v[D];
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c)
+          tmem_ld32(lane_base + tdP + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[c * 32]));
+        tmem_wait_ld();
+        tc_fence_before();
+        mbar_arrive(bar(kDqDrained));
+        if (row < qt.len) {
+          float* dst = prm.dq_acc + ((size_t(qt.start) + row) * prm.Hq + qt.h) * D;
+#pragma unroll
+          for (int i = 0; i < D / 4; ++i)
             red_add_v4(dst + 4 * i, __uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
                        __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
         }
       }
-      tc_fence_before();
-      __syncthreads();
+      gc += un.n_it;
     }
   }
 
-  // ---- epilogue: dK (scaled), dV -> bf16
-  tc_fence_after();
-#pragma unroll 1
-  for (int which = 0; which < 2; ++which) {
-    const uint32_t tsrc = which ? tdK : tdV;
-    __nv_bfloat16* out = which ? prm.dk : prm.dv;
-    const float f = which ? prm.scale : 1.f;
-#pragma unroll 1
-    for (int c = 0; c < D / 32; ++c) {
-      uint32_t v[32];
-      tmem_ld32(lane_base + tsrc + c * 32, v);
-      tmem_wait_ld();
-      if (lane < k_len) {
-        uint4* dst = reinterpret_cast<uint4*>(out + ((size_t(k_start) + lane) * prm.Hkv + kvh) * D + c * 32);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          uint4 w;
-          w.x = pack_bf16(__uint_as_float(v[8 * i + 0]) * f, __uint_as_float(v[8 * i + 1]) * f);
-          w.y = pack_bf16(__uint_as_float(v[8 * i + 2]) * f, __uint_as_float(v[8 * i + 3]) * f);
-          w.z = pack_bf16(__uint_as_float(v[8 * i + 4]) * f, __uint_as_float(v[8 * i + 5]) * f);
-          w.w = pack_bf16(__uint_as_float(v[8 * i + 6]) * f, __uint_as_float(v[8 * i + 7]) * f);
-          dst[i] = w;
-        }
-      }
-    }
-  }
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, kBwdTmemCols);
@@ -318,7 +490,15 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
   bwd_preprocess_kernel<D><<<unsigned((pairs + 7) / 8), 256, 0, stream>>>(
       static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse,
       const_cast<float*>(prm.delta), const_cast<float*>(prm.lse2), int(T), int(Hq));
-  dim3 grid(unsigned(plan->max_tiles) * unsigned(pb.num_kv_heads));
+  static int num_sms = 0;
+  if (!num_sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      num_sms = 148;
+  }
+  const long long units = (long long)plan->max_tiles * pb.num_kv_heads;
+  dim3 grid(unsigned(std::min<long long>(units, num_sms)));
   ProfileEvents& ev = profile_events();
   if (ev.on) cudaEventRecord(ev.bwd0, stream);
   kern<<<grid, kBwdThreads, BwdSmem<D>::kTotal, stream>>>(tq, tk, tv, tdo, prm);
