@@ -82,7 +82,10 @@ bwd_finalize_kernel(const float4* __restrict__ acc, uint2* __restrict__ dq, size
 //   warp 1       MMA issuer (one thread)
 //   warps 2-5    compute warpgroup 0: thread = key row, query columns 0..63 of the tile
 //   warps 6-9    compute warpgroup 1: query columns 64..127
-//   warps 10-13  dQ warpgroup: thread = query row, drains dQ tiles into the fp32 accumulator
+//   warps 10-13  dQ warpgroup: thread = query row; moves each dQ tile from tensor memory
+//                through a swizzled shared-memory staging buffer into the fp32 accumulator
+//                with TMA reduce-add (whole 128-byte lines per row instead of per-thread
+//                16-byte reductions, which saturate the L2 atomic units)
 // Tensor-memory map (columns): [0,128) S^T, overwritten by P^T (bf16: columns [0,32) and
 // [64,96), each warpgroup inside the columns it has read itself); [128,256) dP^T, then the
 // dQ tile; [256,256+D) dV; [384,384+D) dK.
@@ -97,8 +100,8 @@ enum BwdBar : int {
   kKvEmpty,
   kQFullB,       // [2]   33 arrivals: TMA transaction + 32 producer lanes (LSE / Delta)
   kQEmptyB = 4,  // [2]
-  kDoFull = 6,   // [2]
-  kDoEmpty = 8,  // [2]
+  kDoFull = 6,   // dO is single-buffered: free after dV(i), needed again at dP(i+1)
+  kDoEmpty = 8,
   kSFullB = 10,
   kPReady,       // 256
   kDpFull,
@@ -113,9 +116,10 @@ enum BwdBar : int {
 template <int D>
 struct BwdSmem {
   static constexpr int kTileBytes = 128 * D * 2;
+  static constexpr int kStageBytes = 128 * 128;  // one {32 floats x 128 rows} box of a dQ tile
   static constexpr int kK = 0, kV = kTileBytes, kQ = 2 * kTileBytes, kdO = 4 * kTileBytes,
-                       kdS = 6 * kTileBytes, kStats = kdS + 128 * 128 * 2,
-                       kBars = kStats + 2 * 256 * 4;
+                       kStg = 5 * kTileBytes, kdS = kStg + 2 * kStageBytes,
+                       kStats = kdS + 128 * 128 * 2, kBars = kStats + 2 * 256 * 4;
   static constexpr int kUsed = kBars + 8 * kNumBwdBars + 16;
   // The declared 1024-byte alignment of the dynamic shared memory leaves no slack to spend at
   // D = 128 (227 KB limit); the kernel checks the base and reports if it is not aligned.
@@ -163,7 +167,7 @@ template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
            const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
-           BwdParams prm) {
+           const __grid_constant__ CUtensorMap tm_dq, BwdParams prm) {
   using L = BwdSmem<D>;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -202,6 +206,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     tma_prefetch_desc(&tm_k);
     tma_prefetch_desc(&tm_v);
     tma_prefetch_desc(&tm_do);
+    tma_prefetch_desc(&tm_dq);
   }
   if (warp == 0) {
     tmem_alloc(tmem_slot, kBwdTmemCols);
@@ -247,11 +252,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         }
         mbar_arrive(bar(kQFullB + st));
         if (lane == 0) {
-          wait_bar(bar(kDoEmpty + st), par, abort_flag, prm.header, 52);
-          mbar_expect_tx(bar(kDoFull + st), L::kTileBytes);
+          wait_bar(bar(kDoEmpty), (qc & 1) ^ 1, abort_flag, prm.header, 52);
+          mbar_expect_tx(bar(kDoFull), L::kTileBytes);
           for (int b = 0; b < D / 64; ++b)
-            tma_load_3d(sdO + st * L::kTileBytes + b * kBoxBytes, &tm_do, b * 64, qt.h, qt.start,
-                        bar(kDoFull + st));
+            tma_load_3d(sdO + b * kBoxBytes, &tm_do, b * 64, qt.h, qt.start, bar(kDoFull));
         }
       }
     }
@@ -262,12 +266,15 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       constexpr uint32_t idesc_kv = make_idesc(128, D, 0, 1);  // dV, dK : K-major A, MN-major B
       constexpr uint32_t idesc_dq = make_idesc(128, D, 1, 1);  // dQ     : MN-major A and B
       BwdUnit un;
+      const uint64_t dK_k = kmajor_base(sK), dV_k = kmajor_base(sV), dK_mn = mnmajor_base(sK);
+      const uint64_t dS_k = kmajor_base(sdS), dS_mn = mnmajor_base(sdS);
+      constexpr uint64_t kStageStep = uint64_t(L::kTileBytes >> 4);
       auto issue_s = [&](uint32_t st, int q_len) {
         const uint32_t idesc = make_idesc(128, ((q_len + 15) >> 4) << 4, 0, 0);
-        const uint32_t q = sQ + st * L::kTileBytes;
+        const uint64_t dq_k = kmajor_base(sQ) + st * kStageStep;
 #pragma unroll
         for (int k = 0; k < D / 16; ++k)
-          mma_ss(tmem + tS, kmajor_desc(sK, k), kmajor_desc(q, k), idesc, k > 0);
+          mma_ss(tmem + tS, dK_k + kmajor_off(k), dq_k + kmajor_off(k), idesc, k > 0);
         mma_commit(bar(kSFullB));
       };
       for (int rnd = 0; get_bwd_unit(prm, bwd_unit_of_round(rnd), ntiles_total, un); ++rnd, ++ucnt) {
@@ -278,28 +285,31 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         tc_fence_after();
         issue_s(gc & 1, qt.len);
         for (int it = 0; it < un.n_it; ++it) {
-          const uint32_t g = gc + it, st = g & 1, spar = (g >> 1) & 1, par = g & 1;
+          const uint32_t g = gc + it, st = g & 1, par = g & 1;
           const int qsteps = (qt.len + 15) >> 4;
-          const uint32_t q = sQ + st * L::kTileBytes, d_o = sdO + st * L::kTileBytes;
+          const uint64_t dq_mn = mnmajor_base(sQ) + st * kStageStep;
+          const uint64_t ddo_k = kmajor_base(sdO), ddo_mn = mnmajor_base(sdO);
           // dP^T(it) = V dO^T
-          wait_bar(bar(kDoFull + st), spar, abort_flag, prm.header, 62);
+          wait_bar(bar(kDoFull), par, abort_flag, prm.header, 62);
           if (g > 0) wait_bar(bar(kDqDrained), (g - 1) & 1, abort_flag, prm.header, 63);
           tc_fence_after();
           {
             const uint32_t idesc = make_idesc(128, qsteps << 4, 0, 0);
 #pragma unroll
             for (int k = 0; k < D / 16; ++k)
-              mma_ss(tmem + tdP, kmajor_desc(sV, k), kmajor_desc(d_o, k), idesc, k > 0);
+              mma_ss(tmem + tdP, dV_k + kmajor_off(k), ddo_k + kmajor_off(k), idesc, k > 0);
             mma_commit(bar(kDpFull));
           }
           // dV += P^T dO
           wait_bar(bar(kPReady), par, abort_flag, prm.header, 64);
           if (it == 0) wait_bar(bar(kDkvFree), (ucnt & 1) ^ 1, abort_flag, prm.header, 65);
           tc_fence_after();
-          for (int k = 0; k < qsteps; ++k)
-            mma_ts(tmem + tdV, tmem + tS + (k < 4 ? k * 8 : 64 + (k - 4) * 8), mnmajor_desc(d_o, k),
-                   idesc_kv, (it > 0) || (k > 0));
-          mma_commit(bar(kDoEmpty + st));
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            if (k < qsteps)
+              mma_ts(tmem + tdV, tmem + tS + (k < 4 ? k * 8 : 64 + (k - 4) * 8),
+                     ddo_mn + mnmajor_off(k), idesc_kv, (it > 0) || (k > 0));
+          mma_commit(bar(kDoEmpty));
           // S^T(it+1) = K Q^T
           QTile nx = qt;
           if (it + 1 < un.n_it) {
@@ -312,11 +322,16 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           // dQ(it) = dS K, then dK += dS^T Q
           wait_bar(bar(kDsReady), par, abort_flag, prm.header, 67);
           tc_fence_after();
-          for (int k = 0; k < ksteps; ++k)
-            mma_ss(tmem + tdP, mnmajor_desc(sdS, k), mnmajor_desc(sK, k), idesc_dq, k > 0);
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            if (k < ksteps)
+              mma_ss(tmem + tdP, dS_mn + mnmajor_off(k), dK_mn + mnmajor_off(k), idesc_dq, k > 0);
           mma_commit(bar(kDqFull));
-          for (int k = 0; k < qsteps; ++k)
-            mma_ss(tmem + tdK, kmajor_desc(sdS, k), mnmajor_desc(q, k), idesc_kv, (it > 0) || (k > 0));
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            if (k < qsteps)
+              mma_ss(tmem + tdK, dS_k + kmajor_off(k), dq_mn + mnmajor_off(k), idesc_kv,
+                     (it > 0) || (k > 0));
           mma_commit(bar(kQEmptyB + st));
           qt = nx;
         }
@@ -348,12 +363,17 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         tmem_ld32(lane_base + tS + cb + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
         tmem_wait_ld();
         uint32_t pk[32];
+        const float4* sl4 = reinterpret_cast<const float4*>(sl);
         if (full) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float p0 = ex2(fmaf(__uint_as_float(v[2 * i]), prm.scale_log2, -sl[2 * i]));
-            const float p1 = ex2(fmaf(__uint_as_float(v[2 * i + 1]), prm.scale_log2, -sl[2 * i + 1]));
-            pk[i] = pack_bf16(p0, p1);
+          for (int i = 0; i < 16; ++i) {
+            const float4 l = sl4[i];
+            const float p0 = ex2(fmaf(__uint_as_float(v[4 * i]), prm.scale_log2, -l.x));
+            const float p1 = ex2(fmaf(__uint_as_float(v[4 * i + 1]), prm.scale_log2, -l.y));
+            const float p2 = ex2(fmaf(__uint_as_float(v[4 * i + 2]), prm.scale_log2, -l.z));
+            const float p3 = ex2(fmaf(__uint_as_float(v[4 * i + 3]), prm.scale_log2, -l.w));
+            pk[2 * i] = pack_bf16(p0, p1);
+            pk[2 * i + 1] = pack_bf16(p2, p3);
           }
         } else {
           // visible iff the key row exists, the query column exists, and (diagonal tile) the
@@ -386,8 +406,9 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           for (int i = 0; i < 16; ++i) {
             const uint32_t pp = pk[16 * half + i];
             const float p0 = __uint_as_float(pp << 16), p1 = __uint_as_float(pp & 0xffff0000u);
-            float d0 = p0 * (__uint_as_float(d[2 * i]) - sl[128 + 32 * half + 2 * i]);
-            float d1 = p1 * (__uint_as_float(d[2 * i + 1]) - sl[128 + 32 * half + 2 * i + 1]);
+            const float2 dl = reinterpret_cast<const float2*>(sl + 128 + 32 * half)[i];
+            float d0 = p0 * (__uint_as_float(d[2 * i]) - dl.x);
+            float d1 = p1 * (__uint_as_float(d[2 * i + 1]) - dl.y);
             if (!full) {  // stale tensor-memory columns may hold anything
               d0 = (pp & 0xffffu) ? d0 : 0.f;
               d1 = (pp & 0xffff0000u) ? d1 : 0.f;
@@ -436,8 +457,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   } else {
     // ------------------------------------------------------------ dQ warpgroup
     const int row = 32 * (warp & 3) + lane;
+    const bool leader = (warp == 10 && lane == 0);
     const uint32_t lane_base = tmem + (uint32_t(32 * (warp & 3)) << 16);
-    uint32_t gc = 0;
+    const uint32_t stg = base + L::kStg;
+    uint32_t gc = 0, chunk = 0;
     BwdUnit un;
     for (int rnd = 0; get_bwd_unit(prm, bwd_unit_of_round(rnd), ntiles_total, un); ++rnd) {
       for (int it = 0; it < un.n_it; ++it) {
@@ -445,23 +468,42 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         const uint32_t g = gc + it;
         wait_bar(bar(kDqFull), g & 1, abort_flag, prm.header, 80);
         tc_fence_after();
-        uint32_t v[D];
+#pragma unroll 1
+        for (int c = 0; c < D / 32; ++c, ++chunk) {
+          const uint32_t buf = stg + (chunk & 1) * L::kStageBytes;
+          // the reduce issued two chunks ago must have finished reading this buffer
+          if (leader) bulk_wait_group_read<1>();
+          named_barrier_sync(1, 128);
+          uint32_t w[32];
+          tmem_ld32(lane_base + tdP + c * 32, w);
+          tmem_wait_ld();
+          if (c == D / 32 - 1) {
+            tc_fence_before();
+            mbar_arrive(bar(kDqDrained));
+          }
+          if (row >= qt.len) {  // rows past the tile's end belong to other tokens: add zero
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c)
-          tmem_ld32(lane_base + tdP + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[c * 32]));
-        tmem_wait_ld();
-        tc_fence_before();
-        mbar_arrive(bar(kDqDrained));
-        if (row < qt.len) {
-          float* dst = prm.dq_acc + ((size_t(qt.start) + row) * prm.Hq + qt.h) * D;
+            for (int i = 0; i < 32; ++i) w[i] = 0u;
+          }
+          const uint32_t row_addr = buf + row * 128;
 #pragma unroll
-          for (int i = 0; i < D / 4; ++i)
-            red_add_v4(dst + 4 * i, __uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
-                       __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+          for (int i = 0; i < 8; ++i) {
+            const uint32_t ch = uint32_t(i) ^ uint32_t(row & 7);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + ch * 16),
+                         "r"(w[4 * i]), "r"(w[4 * i + 1]), "r"(w[4 * i + 2]), "r"(w[4 * i + 3])
+                         : "memory");
+          }
+          fence_proxy_async_smem();
+          named_barrier_sync(1, 128);
+          if (leader) {
+            tma_reduce_add_3d(&tm_dq, buf, c * 32, qt.h, qt.start);
+            bulk_commit_group();
+          }
         }
       }
       gc += un.n_it;
     }
+    if (leader) bulk_wait_group<0>();
   }
 
   tc_fence_before();
@@ -472,8 +514,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 template <int D>
 cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, const void* d_o,
                          void* dq, const CUtensorMap& tq, const CUtensorMap& tk,
-                         const CUtensorMap& tv, const CUtensorMap& tdo, const BwdParams& prm,
-                         cudaStream_t stream, int* launches) {
+                         const CUtensorMap& tv, const CUtensorMap& tdo, const CUtensorMap& tdq,
+                         const BwdParams& prm, cudaStream_t stream, int* launches) {
   static bool configured = false;
   auto kern = bwd_kernel<D>;
   if (!configured) {
@@ -501,7 +543,7 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
   dim3 grid(unsigned(std::min<long long>(units, num_sms)));
   ProfileEvents& ev = profile_events();
   if (ev.on) cudaEventRecord(ev.bwd0, stream);
-  kern<<<grid, kBwdThreads, BwdSmem<D>::kTotal, stream>>>(tq, tk, tv, tdo, prm);
+  kern<<<grid, kBwdThreads, BwdSmem<D>::kTotal, stream>>>(tq, tk, tv, tdo, tdq, prm);
   if (ev.on) {
     cudaEventRecord(ev.bwd1, stream);
     ev.bwd_valid = true;
@@ -542,9 +584,12 @@ cudaError_t launch_bwd(const pp_plan* plan, const void* q, const void* k, const 
   prm.Hkv = pb.num_kv_heads;
   prm.scale = scale;
   prm.scale_log2 = scale * 1.4426950408889634f;
+  CUtensorMap tdq;
+  if (!encode_thd_f32(&tdq, prm.dq_acc, pb.total_tokens, pb.num_q_heads, pb.head_dim))
+    return cudaErrorNotSupported;
   return pb.head_dim == 128
-             ? launch_bwd_t<128>(plan, o, lse, d_o, dq, tq, tk, tv, tdo, prm, stream, launches)
-             : launch_bwd_t<64>(plan, o, lse, d_o, dq, tq, tk, tv, tdo, prm, stream, launches);
+             ? launch_bwd_t<128>(plan, o, lse, d_o, dq, tq, tk, tv, tdo, tdq, prm, stream, launches)
+             : launch_bwd_t<64>(plan, o, lse, d_o, dq, tq, tk, tv, tdo, tdq, prm, stream, launches);
 }
 
 // ---------------------------------------------------------------- built-in scratch

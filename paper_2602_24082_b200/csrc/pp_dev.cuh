@@ -59,6 +59,20 @@ inline bool encode_thd(CUtensorMap* m, const void* base, int T, int H, int D, in
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// fp32 tensor [T][H][D] for TMA reductions: one box = 32 floats x 1 head x 128 tokens,
+// 128-byte swizzled (row r at r * 128 bytes, 16-byte chunks XOR-ed with r mod 8).
+inline bool encode_thd_f32(CUtensorMap* m, const void* base, int T, int H, int D) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {cuuint64_t(D), cuuint64_t(H), cuuint64_t(T)};
+  cuuint64_t strides[2] = {cuuint64_t(D) * 4, cuuint64_t(H) * D * 4};
+  cuuint32_t box[3] = {32, 1, 128};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box,
+            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 constexpr uint32_t kBoxBytes = 128 * 128;  // one {64 x 128 rows} bf16 box
 
 // K-major operand descriptor for k-step `k16` (16 elements of the contraction = 32 bytes
@@ -71,5 +85,19 @@ __device__ __forceinline__ uint64_t kmajor_desc(uint32_t tile_base, int k16) {
 __device__ __forceinline__ uint64_t mnmajor_desc(uint32_t tile_base, int k16) {
   return make_sdesc(tile_base + k16 * 2048, kBoxBytes, 1024);
 }
+
+// Descriptor arithmetic for unrolled k-loops: a descriptor for k-step k16 is the tile's base
+// descriptor plus a compile-time constant in its address field (shared-memory addresses stay
+// below 2^18, so the 14-bit field cannot overflow).
+__device__ __forceinline__ uint64_t kmajor_base(uint32_t tile_base) {
+  return make_sdesc(tile_base, 16, 1024);
+}
+__device__ __forceinline__ uint64_t mnmajor_base(uint32_t tile_base) {
+  return make_sdesc(tile_base, kBoxBytes, 1024);
+}
+__host__ __device__ constexpr uint64_t kmajor_off(int k16) {
+  return uint64_t(((k16 >> 2) * kBoxBytes + (k16 & 3) * 32) >> 4);
+}
+__host__ __device__ constexpr uint64_t mnmajor_off(int k16) { return uint64_t((k16 * 2048) >> 4); }
 
 }  // namespace pp
