@@ -153,12 +153,21 @@ struct QTile {
   bool diag;
 };
 
-__device__ __forceinline__ QTile q_tile_of(const BwdParams& prm, const BwdUnit& un, int it) {
+// (head, query tile) position inside a unit, advanced without divisions
+struct QIter {
+  int hh = 0, qt = 0;
+};
+__device__ __forceinline__ void q_advance(QIter& s, int nq) {
+  if (++s.qt == nq) {
+    s.qt = 0;
+    ++s.hh;
+  }
+}
+__device__ __forceinline__ QTile q_tile_at(const BwdParams& prm, const BwdUnit& un, const QIter& s) {
   QTile q;
-  const int hh = it / un.nq, qt = it - hh * un.nq;
-  q.h = un.kvh * (prm.Hq / prm.Hkv) + hh;
-  q.diag = (qt == 0);
-  q.start = q.diag ? un.tile.start : un.tile.start + un.tile.len + (qt - 1) * kTile;
+  q.h = un.kvh * (prm.Hq / prm.Hkv) + s.hh;
+  q.diag = (s.qt == 0);
+  q.start = q.diag ? un.tile.start : un.tile.start + un.tile.len + (s.qt - 1) * kTile;
   q.len = q.diag ? un.tile.len : min(kTile, un.tile.vis_end - q.start);
   return q;
 }
@@ -231,9 +240,20 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           tma_load_3d(sV + b * kBoxBytes, &tm_v, b * 64, un.kvh, un.tile.start, bar(kKvFull));
         }
       }
-      for (int it = 0; it < un.n_it; ++it, ++qc) {
-        const QTile qt = q_tile_of(prm, un, it);
+      QIter qi;
+      for (int it = 0; it < un.n_it; ++it, ++qc, q_advance(qi, un.nq)) {
+        const QTile qt = q_tile_at(prm, un, qi);
         const uint32_t st = qc & 1, par = ((qc >> 1) & 1) ^ 1;
+        // per-query statistics, fetched before the stage is known to be free;
+        // +inf LSE and zero Delta switch off columns past the tile's end
+        const size_t row0 = size_t(qt.h) * prm.T + qt.start;
+        float r_lse[4], r_del[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int c = lane + 32 * i;
+          r_lse[i] = c < qt.len ? prm.lse2[row0 + c] : INFINITY;
+          r_del[i] = c < qt.len ? prm.delta[row0 + c] : 0.f;
+        }
         wait_bar(bar(kQEmptyB + st), par, abort_flag, prm.header, 51);
         if (lane == 0) {
           mbar_expect_tx(bar(kQFullB + st), L::kTileBytes);
@@ -241,14 +261,11 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             tma_load_3d(sQ + st * L::kTileBytes + b * kBoxBytes, &tm_q, b * 64, qt.h, qt.start,
                         bar(kQFullB + st));
         }
-        // per-query statistics; +inf LSE and zero Delta switch off columns past the tile's end
         float* sl = stats + st * 256;
-        const size_t row0 = size_t(qt.h) * prm.T + qt.start;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const int c = lane + 32 * i;
-          sl[c] = c < qt.len ? prm.lse2[row0 + c] : INFINITY;
-          sl[128 + c] = c < qt.len ? prm.delta[row0 + c] : 0.f;
+          sl[lane + 32 * i] = r_lse[i];
+          sl[128 + lane + 32 * i] = r_del[i];
         }
         mbar_arrive(bar(kQFullB + st));
         if (lane == 0) {
@@ -280,7 +297,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       for (int rnd = 0; get_bwd_unit(prm, bwd_unit_of_round(rnd), ntiles_total, un); ++rnd, ++ucnt) {
         const int ksteps = (un.tile.len + 15) >> 4;
         wait_bar(bar(kKvFull), ucnt & 1, abort_flag, prm.header, 60);
-        QTile qt = q_tile_of(prm, un, 0);
+        QIter qi;
+        QTile qt = q_tile_at(prm, un, qi);
         wait_bar(bar(kQFullB + (gc & 1)), (gc >> 1) & 1, abort_flag, prm.header, 61);
         tc_fence_after();
         issue_s(gc & 1, qt.len);
@@ -313,7 +331,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           // S^T(it+1) = K Q^T
           QTile nx = qt;
           if (it + 1 < un.n_it) {
-            nx = q_tile_of(prm, un, it + 1);
+            q_advance(qi, un.nq);
+            nx = q_tile_at(prm, un, qi);
             const uint32_t g1 = g + 1;
             wait_bar(bar(kQFullB + (g1 & 1)), (g1 >> 1) & 1, abort_flag, prm.header, 66);
             tc_fence_after();
@@ -350,8 +369,9 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     BwdUnit un;
     for (int rnd = 0; get_bwd_unit(prm, bwd_unit_of_round(rnd), ntiles_total, un); ++rnd, ++ucnt) {
       const bool row_ok = row < un.tile.len;
-      for (int it = 0; it < un.n_it; ++it) {
-        const QTile qt = q_tile_of(prm, un, it);
+      QIter qi;
+      for (int it = 0; it < un.n_it; ++it, q_advance(qi, un.nq)) {
+        const QTile qt = q_tile_at(prm, un, qi);
         const uint32_t g = gc + it, st = g & 1, par = g & 1;
         const float* sl = stats + st * 256 + cb;
         const bool full = !qt.diag && qt.len == kTile && un.tile.len == kTile;
@@ -463,8 +483,9 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     uint32_t gc = 0, chunk = 0;
     BwdUnit un;
     for (int rnd = 0; get_bwd_unit(prm, bwd_unit_of_round(rnd), ntiles_total, un); ++rnd) {
-      for (int it = 0; it < un.n_it; ++it) {
-        const QTile qt = q_tile_of(prm, un, it);
+      QIter qi;
+      for (int it = 0; it < un.n_it; ++it, q_advance(qi, un.nq)) {
+        const QTile qt = q_tile_at(prm, un, qi);
         const uint32_t g = gc + it;
         wait_bar(bar(kDqFull), g & 1, abort_flag, prm.header, 80);
         tc_fence_after();

@@ -13,11 +13,29 @@ constexpr uint32_t kSpinLimit = 1u << 21;  // polls of mbarrier.try_wait before 
 // Waits for a phase of an mbarrier, but never forever: after kSpinLimit polls the CTA records
 // the site in the plan's status word, raises its abort flag (which turns every later wait of
 // this CTA into a no-op) and carries on to its normal exit path.
+#ifdef PP_TIMING
+// Developer switch (-DPP_TIMING): cycles CTA 0 spends in each wait site, summed over lane 0
+// of every warp that waits there; slot 127 holds CTA 0's total cycles.
+static __device__ unsigned long long g_wait_cycles[128];
+#endif
+
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                          int32_t* header, int site) {
+#ifndef PP_TIMING
+  if (mbar_try_wait(bar, parity)) return true;  // fast path: already complete
+#endif
   if (*abort_flag) return false;
+#ifdef PP_TIMING
+  const long long t0 = clock64();
+#endif
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait(bar, parity)) {
+#ifdef PP_TIMING
+      if (blockIdx.x == 0 && (threadIdx.x & 31) == 0)
+        atomicAdd(&g_wait_cycles[site & 127], (unsigned long long)(clock64() - t0));
+#endif
+      return true;
+    }
     if ((it & 0xfff) == 0xfff && *abort_flag) return false;
   }
   if (atomicCAS(&header[0], kStatusOk, kStatusWaitExpired) == kStatusOk) header[1] = site;
