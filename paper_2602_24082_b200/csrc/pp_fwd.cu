@@ -186,12 +186,15 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       uint32_t kc = 0, vc = 0, tc[2] = {0, 0}, uc[2] = {0, 0};
       constexpr uint32_t idesc_o = make_idesc(128, D, 0, 1);
       Unit un;
+      const uint64_t dq0 = kmajor_base(sQ), dk0 = kmajor_base(sK), dv0 = mnmajor_base(sV);
+      constexpr uint64_t kStageStep = uint64_t(L::kTileBytes >> 4);
       auto issue_qk = [&](int s, uint32_t kstage, int k_len) {
-        const uint32_t idesc_s = make_idesc(128, ((k_len + 15) >> 4) << 4, 0, 0);
-        const uint32_t q = sQ + s * L::kTileBytes, k = sK + kstage * L::kTileBytes;
+        const uint32_t idesc_s = k_len == kTile ? make_idesc(128, 128, 0, 0)
+                                                : make_idesc(128, ((k_len + 15) >> 4) << 4, 0, 0);
+        const uint64_t dq = dq0 + s * kStageStep, dk = dk0 + kstage * kStageStep;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk)
-          mma_ss(tmem + s * 128, kmajor_desc(q, kk), kmajor_desc(k, kk), idesc_s, kk > 0);
+          mma_ss(tmem + s * 128, dq + kmajor_off(kk), dk + kmajor_off(kk), idesc_s, kk > 0);
         mma_commit(bar(kSFull + s));
       };
       for (int rnd = 0; get_unit(prm, unit_of_round(rnd), ntiles_total, un); ++rnd) {
@@ -214,15 +217,17 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           wait_bar(bar(kVFull + (vc & 1)), (vc >> 1) & 1, abort_flag, prm.header, 33);
           if (has_next)
             wait_bar(bar(kKFull + (kc & 1)), (kc >> 1) & 1, abort_flag, prm.header, 34);
-          const uint32_t vbase = sV + (vc & 1) * L::kTileBytes;
+          const uint64_t dv = dv0 + (vc & 1) * kStageStep;
           for (int s = 0; s < un.nslots; ++s) {
             wait_bar(bar(kPFull + s), tc[s] & 1, abort_flag, prm.header, 35 + s);
             if (j == 0) wait_bar(bar(kOFree + s), (uc[s] & 1) ^ 1, abort_flag, prm.header, 37 + s);
             tc_fence_after();
             const int ksteps = (cur_len + 15) >> 4;
-            for (int kk = 0; kk < ksteps; ++kk)
-              mma_ts(tmem + 256 + s * 128, tmem + s * 128 + kk * 8, mnmajor_desc(vbase, kk), idesc_o,
-                     (j > 0) || (kk > 0));
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk)
+              if (kk < ksteps)
+                mma_ts(tmem + 256 + s * 128, tmem + s * 128 + kk * 8, dv + mnmajor_off(kk), idesc_o,
+                       (j > 0) || (kk > 0));
             mma_commit(bar(kODone + s));
             ++tc[s];
             if (has_next) {
