@@ -223,10 +223,11 @@ def run_ours(args):
 
     def step():
         plan = B.pp_build_plan(desc, Hq, Hkv, D, T, dev, device_arrays=desc_dev, workspace=ws)
+        n = B.pp_last_launch_count()
         if "scratch" in plan_holder:
             plan._bwd_scratch = plan_holder["scratch"]
         B.pp_attn_fwd(plan, q, k, v, scale, o=o, lse=lse)
-        n = 4 + B.pp_last_launch_count()
+        n += B.pp_last_launch_count()
         B.pp_attn_bwd(plan, q, k, v, o, lse, do, scale, d_q=dq, d_k=dk, d_v=dv)
         n += B.pp_last_launch_count()
         plan_holder["scratch"] = plan.bwd_scratch()

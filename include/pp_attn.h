@@ -154,8 +154,8 @@ int pp_attn_bwd_noalloc(const pp_plan* plan, const void* q, const void* k, const
                         const void* o, const float* lse, const void* d_o, float softmax_scale,
                         void* d_q, void* d_k, void* d_v, pp_stream_t stream);
 
-/* Kernel launches enqueued by the last pp_attn_fwd / pp_attn_bwd / pp_attn_step_host call of
- * this thread. */
+/* Kernel launches enqueued by the last pp_build_plan / pp_attn_fwd / pp_attn_bwd /
+ * pp_attn_bwd_noalloc / pp_attn_step_host call of this thread. */
 int pp_last_launch_count(void);
 
 /*

@@ -110,7 +110,8 @@ int pp_build_plan(const pp_problem* problem, void* d_workspace, size_t workspace
     plan->prob.grp_resp_off = dst[2];
     plan->prob.resp_len = dst[3];
   }
-  if (pp::launch_plan(plan, s) != cudaSuccess) {
+  g_last_launches = 0;
+  if (pp::launch_plan(plan, s, &g_last_launches) != cudaSuccess) {
     delete plan;
     return PP_ERR_CUDA;
   }
@@ -255,7 +256,7 @@ int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_
   pp_plan* plan = nullptr;
   rc = pp_build_plan(problem, base + a.plan, a.scratch - a.plan, stream, &plan);
   if (rc) return rc;
-  int launches = 4;
+  int launches = g_last_launches;
   rc = pp_attn_fwd(plan, base + a.q, base + a.k, base + a.v, softmax_scale, base + a.o,
                    reinterpret_cast<float*>(base + a.lse), nullptr, 0, stream);
   launches += g_last_launches;

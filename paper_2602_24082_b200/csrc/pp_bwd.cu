@@ -34,30 +34,42 @@ struct BwdParams {
 };
 
 // ---------------------------------------------------------------- preprocess
+// One warp per (token, query head) row: Delta = sum_d dO * O, the LSE in base-2 units, and the
+// row of the fp32 dQ accumulator cleared (so no separate memset pass over it is needed).
 template <int D>
 __global__ void __launch_bounds__(256)
 bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
                       const float* __restrict__ lse, float* __restrict__ delta,
-                      float* __restrict__ lse2, int T, int Hq) {
+                      float* __restrict__ lse2, float* __restrict__ dq_acc, int T, int Hq) {
   const int lane = threadIdx.x & 31;
-  const long long idx = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (idx >= (long long)T * Hq) return;
-  const int t = int(idx / Hq), h = int(idx % Hq);
-  constexpr int kPer = D / 32;  // elements per lane: 4 (D=128) or 2 (D=64)
-  const __nv_bfloat16* po = o + idx * D + lane * kPer;
-  const __nv_bfloat16* pd = d_o + idx * D + lane * kPer;
-  float acc = 0.f;
+  const long long rows = (long long)T * Hq;
+  const long long stride = (long long)gridDim.x * 8;
+  for (long long idx = (long long)blockIdx.x * 8 + (threadIdx.x >> 5); idx < rows; idx += stride) {
+    const int t = int(idx / Hq), h = int(idx - (long long)t * Hq);
+    float acc = 0.f;
+    if (D == 128) {
+      const uint2 a = reinterpret_cast<const uint2*>(o + idx * D)[lane];
+      const uint2 b = reinterpret_cast<const uint2*>(d_o + idx * D)[lane];
+      const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a.x));
+      const float2 a1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a.y));
+      const float2 b0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b.x));
+      const float2 b1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b.y));
+      acc = a0.x * b0.x + a0.y * b0.y + a1.x * b1.x + a1.y * b1.y;
+      reinterpret_cast<float4*>(dq_acc + idx * D)[lane] = make_float4(0.f, 0.f, 0.f, 0.f);
+    } else {
+      const uint32_t a = reinterpret_cast<const uint32_t*>(o + idx * D)[lane];
+      const uint32_t b = reinterpret_cast<const uint32_t*>(d_o + idx * D)[lane];
+      const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a));
+      const float2 b0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b));
+      acc = a0.x * b0.x + a0.y * b0.y;
+      reinterpret_cast<float2*>(dq_acc + idx * D)[lane] = make_float2(0.f, 0.f);
+    }
 #pragma unroll
-  for (int i = 0; i < kPer; i += 2) {
-    float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(po + i));
-    float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(pd + i));
-    acc += a.x * b.x + a.y * b.y;
-  }
-#pragma unroll
-  for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
-  if (lane == 0) {
-    delta[size_t(h) * T + t] = acc;
-    lse2[size_t(h) * T + t] = lse[size_t(h) * T + t] * 1.4426950408889634f;
+    for (int sft = 16; sft > 0; sft >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sft);
+    if (lane == 0) {
+      delta[size_t(h) * T + t] = acc;
+      lse2[size_t(h) * T + t] = lse[size_t(h) * T + t] * 1.4426950408889634f;
+    }
   }
 }
 
@@ -547,12 +559,11 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
   }
   const pp_problem& pb = plan->prob;
   const size_t T = pb.total_tokens, Hq = pb.num_q_heads;
-  cudaError_t e = cudaMemsetAsync(prm.dq_acc, 0, 4 * T * Hq * D, stream);
-  if (e != cudaSuccess) return e;
   const long long pairs = (long long)T * Hq;
-  bwd_preprocess_kernel<D><<<unsigned((pairs + 7) / 8), 256, 0, stream>>>(
+  const unsigned pre_blocks = unsigned(std::min<long long>((pairs + 7) / 8, 148 * 32));
+  bwd_preprocess_kernel<D><<<pre_blocks, 256, 0, stream>>>(
       static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse,
-      const_cast<float*>(prm.delta), const_cast<float*>(prm.lse2), int(T), int(Hq));
+      const_cast<float*>(prm.delta), const_cast<float*>(prm.lse2), prm.dq_acc, int(T), int(Hq));
   static int num_sms = 0;
   if (!num_sms) {
     int dev = 0;

@@ -130,7 +130,7 @@ bool profile_enable(bool on);
 bool profile_read(float* fwd_ms, float* bwd_ms);
 
 // launchers (defined in the .cu files); all return a cudaError_t
-cudaError_t launch_plan(const pp_plan* plan, cudaStream_t stream);
+cudaError_t launch_plan(const pp_plan* plan, cudaStream_t stream, int* launches);
 cudaError_t launch_fwd(const pp_plan* plan, const void* q, const void* k, const void* v, float scale,
                        void* o, float* lse, cudaStream_t stream, int* launches);
 cudaError_t launch_bwd(const pp_plan* plan, const void* q, const void* k, const void* v,

@@ -33,8 +33,9 @@ __device__ __forceinline__ void set_status(int32_t* header, int32_t status, int3
 // Segment order: group 0 prompt, group 0 responses, group 1 prompt, ...  so the prompt of
 // group g is segment g + resp_off[g] and response x (global index) of group g is g + 1 + x.
 
-// One block.  Validates, writes segment lengths, scans them into seg_start / seg_tile0.
-__global__ void __launch_bounds__(1024) plan_scan_kernel(PlanPtrs p) {
+// One block of 1024 threads.  Validates, writes segment lengths, scans them into seg_start /
+// seg_tile0.  Returns (uniformly) whether the descriptors were accepted.
+__device__ __forceinline__ bool plan_scan_body(const PlanPtrs& p) {
   __shared__ int32_t s_tok[1024];
   __shared__ int32_t s_til[1024];
   __shared__ int32_t s_carry[2];
@@ -71,7 +72,7 @@ __global__ void __launch_bounds__(1024) plan_scan_kernel(PlanPtrs p) {
     }
   }
   __syncthreads();
-  if (p.header[0] != kStatusOk) return;
+  if (p.header[0] != kStatusOk) return false;
 
   // chunked exclusive scan of lengths and tile counts
   for (int base = 0; base < p.nseg; base += blockDim.x) {
@@ -112,7 +113,11 @@ __global__ void __launch_bounds__(1024) plan_scan_kernel(PlanPtrs p) {
       p.header[2] = s_carry[1];  // number of tiles
     }
   }
+  __syncthreads();
+  return p.header[0] == kStatusOk;
 }
+
+__global__ void __launch_bounds__(1024) plan_scan_kernel(PlanPtrs p) { plan_scan_body(p); }
 
 // largest s in [0, n) with a[s] <= x  (a is non-decreasing, a[0] <= x)
 __device__ __forceinline__ int upper_segment(const int32_t* a, int n, int x) {
@@ -134,11 +139,7 @@ __device__ __forceinline__ int group_of_segment(const PlanPtrs& p, int s) {
   return lo;
 }
 
-__global__ void plan_tiles_kernel(PlanPtrs p) {
-  if (p.header[0] != kStatusOk) return;
-  const int ntiles = p.header[2];
-  int t = blockIdx.x * blockDim.x + threadIdx.x;
-  if (t >= ntiles) return;
+__device__ __forceinline__ void plan_tile_body(const PlanPtrs& p, int t) {
   int s = upper_segment(p.seg_tile0, p.nseg, t);
   // segments with zero tiles cannot exist (len >= 1), so seg_tile0 is strictly increasing
   int g = group_of_segment(p, s);
@@ -164,14 +165,23 @@ __global__ void plan_tiles_kernel(PlanPtrs p) {
   p.tiles[t] = tl;
 }
 
-__global__ void plan_key_end_kernel(PlanPtrs p) {
+__global__ void plan_tiles_kernel(PlanPtrs p) {
   if (p.header[0] != kStatusOk) return;
-  int j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= p.T) return;
+  int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t < p.header[2]) plan_tile_body(p, t);
+}
+
+__device__ __forceinline__ void plan_key_end_body(const PlanPtrs& p, int j) {
   int s = upper_segment(p.seg_start, p.nseg, j);
   int g = group_of_segment(p, s);
   bool prompt = (s == g + p.grp_resp_off[g]);
   p.key_end[j] = prompt ? p.seg_start[(g + 1) + p.grp_resp_off[g + 1]] : p.seg_start[s + 1];
+}
+
+__global__ void plan_key_end_kernel(PlanPtrs p) {
+  if (p.header[0] != kStatusOk) return;
+  int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j < p.T) plan_key_end_body(p, j);
 }
 
 __device__ __forceinline__ int bwd_work(const Tile& t) {
@@ -179,11 +189,7 @@ __device__ __forceinline__ int bwd_work(const Tile& t) {
 }
 
 // Longest-work-first orders by rank counting (tile counts are small: T/128 + segments).
-__global__ void plan_order_kernel(PlanPtrs p) {
-  if (p.header[0] != kStatusOk) return;
-  const int n = p.header[2];
-  int t = blockIdx.x * blockDim.x + threadIdx.x;
-  if (t >= n) return;
+__device__ __forceinline__ void plan_order_body(const PlanPtrs& p, int t, int n) {
   Tile me = p.tiles[t];
   int wf = me.work, wb = bwd_work(me);
   int rf = 0, rb = 0;
@@ -195,6 +201,24 @@ __global__ void plan_order_kernel(PlanPtrs p) {
   }
   p.fwd_order[rf] = t;
   p.bwd_order[rb] = t;
+}
+
+__global__ void plan_order_kernel(PlanPtrs p) {
+  if (p.header[0] != kStatusOk) return;
+  const int n = p.header[2];
+  int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t < n) plan_order_body(p, t, n);
+}
+
+// The whole plan in one block: used when the problem is small enough that one block's
+// latency beats four dependent launches (every stage only needs block-level ordering).
+__global__ void __launch_bounds__(1024) plan_fused_kernel(PlanPtrs p) {
+  if (!plan_scan_body(p)) return;
+  const int n = p.header[2];
+  for (int t = threadIdx.x; t < n; t += blockDim.x) plan_tile_body(p, t);
+  for (int j = threadIdx.x; j < p.T; j += blockDim.x) plan_key_end_body(p, j);
+  __syncthreads();
+  for (int t = threadIdx.x; t < n; t += blockDim.x) plan_order_body(p, t, n);
 }
 
 }  // namespace
@@ -229,7 +253,7 @@ bool profile_read(float* fwd_ms, float* bwd_ms) {
   return ok;
 }
 
-cudaError_t launch_plan(const pp_plan* plan, cudaStream_t stream) {
+cudaError_t launch_plan(const pp_plan* plan, cudaStream_t stream, int* launches) {
   PlanPtrs p;
   char* ws = plan->ws;
   const PlanLayout& l = plan->lay;
@@ -251,11 +275,17 @@ cudaError_t launch_plan(const pp_plan* plan, cudaStream_t stream) {
   p.nseg = plan->nseg;
   p.max_tiles = plan->max_tiles;
 
-  plan_scan_kernel<<<1, 1024, 0, stream>>>(p);
   int mt = plan->max_tiles;
+  if (mt <= 2048 && p.T <= (1 << 18)) {
+    plan_fused_kernel<<<1, 1024, 0, stream>>>(p);
+    if (launches) *launches = 1;
+    return cudaGetLastError();
+  }
+  plan_scan_kernel<<<1, 1024, 0, stream>>>(p);
   plan_tiles_kernel<<<(mt + 255) / 256, 256, 0, stream>>>(p);
   plan_key_end_kernel<<<(p.T + 255) / 256, 256, 0, stream>>>(p);
   plan_order_kernel<<<(mt + 127) / 128, 128, 0, stream>>>(p);
+  if (launches) *launches = 4;
   return cudaGetLastError();
 }
 
