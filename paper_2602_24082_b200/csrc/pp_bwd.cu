@@ -195,6 +195,9 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 
   if (prm.header[0] != kStatusOk) return;
   const int ntiles_total = prm.header[2];
+#ifdef PP_TIMING
+  const long long t_kernel0 = clock64();
+#endif
 
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -542,7 +545,30 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, kBwdTmemCols);
+#ifdef PP_TIMING
+  if (blockIdx.x == 0 && tid == 0) g_wait_cycles[127] = (unsigned long long)(clock64() - t_kernel0);
+  if (tid == 0) g_cta_cycles[blockIdx.x & 255] = (unsigned long long)(clock64() - t_kernel0);
+#endif
 }
+
+#ifdef PP_TIMING
+}  // namespace
+}  // namespace pp
+extern "C" int pp_debug_bwd_cta_cycles(unsigned long long* out) {
+  return cudaMemcpyFromSymbol(out, pp::g_cta_cycles, sizeof(unsigned long long) * 256) == cudaSuccess ? 0 : -5;
+}
+extern "C" int pp_debug_bwd_wait_cycles(unsigned long long* out, int reset) {
+  if (out && cudaMemcpyFromSymbol(out, pp::g_wait_cycles, sizeof(unsigned long long) * 128) != cudaSuccess)
+    return -5;
+  if (reset) {
+    static unsigned long long zeros[128] = {};
+    if (cudaMemcpyToSymbol(pp::g_wait_cycles, zeros, sizeof zeros) != cudaSuccess) return -5;
+  }
+  return 0;
+}
+namespace pp {
+namespace {
+#endif
 
 template <int D>
 cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, const void* d_o,

@@ -17,6 +17,7 @@ constexpr uint32_t kSpinLimit = 1u << 21;  // polls of mbarrier.try_wait before 
 // Developer switch (-DPP_TIMING): cycles CTA 0 spends in each wait site, summed over lane 0
 // of every warp that waits there; slot 127 holds CTA 0's total cycles.
 static __device__ unsigned long long g_wait_cycles[128];
+static __device__ unsigned long long g_cta_cycles[256];  // per-CTA busy cycles
 #endif
 
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag,

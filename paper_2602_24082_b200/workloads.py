@@ -160,6 +160,41 @@ def slice_heads(w: Workload, tens, row_ids: Sequence[int], kv_heads: Sequence[in
     return sub, (sq, sk, sv, sdo), tok, qh
 
 
+def slice_groups(w: Workload, tens, groups: Sequence[Tuple[int, int]], kv_heads: Sequence[int]):
+    """Independent sub-problem made of whole groups (row, index-in-row) and KV heads with all
+    their query heads; each selected group becomes a row of its own.  Attention never crosses
+    a group, so the sub-problem's results equal the corresponding slice of the full results.
+
+    Returns (sub_workload, (q, k, v, do), token_index, q_head_index)."""
+    r = w.num_q_heads // w.num_kv_heads
+    offs = w.row_offsets()
+    rows, tok, lv, new_off = [], [], [], 0
+    for (ri, gi) in groups:
+        t0 = offs[ri] + sum(p + sum(rs) for (p, rs) in w.rows[ri][:gi])
+        p, rs = w.rows[ri][gi]
+        L = p + sum(rs)
+        rows.append([(p, tuple(rs))])
+        tok.append(torch.arange(t0, t0 + L))
+        for (lo, hi) in w.low_var_ranges:
+            a, b = max(lo, t0), min(hi, t0 + L)
+            if a < b:
+                lv.append((a - t0 + new_off, b - t0 + new_off))
+        new_off += L
+    tok = torch.cat(tok)
+    qh = torch.tensor([c * r + i for c in kv_heads for i in range(r)], dtype=torch.long)
+    kh = torch.tensor(list(kv_heads), dtype=torch.long)
+    q, k, v, do = tens
+    dev = q.device
+    tok_d, qh_d, kh_d = tok.to(dev), qh.to(dev), kh.to(dev)
+    sub = dataclasses.replace(w, name=w.name + f"/groups{list(groups)}", rows=rows,
+                              num_q_heads=len(qh), num_kv_heads=len(kh), low_var_ranges=lv)
+    sq = q.index_select(0, tok_d).index_select(1, qh_d).contiguous()
+    sk = k.index_select(0, tok_d).index_select(1, kh_d).contiguous()
+    sv = v.index_select(0, tok_d).index_select(1, kh_d).contiguous()
+    sdo = do.index_select(0, tok_d).index_select(1, qh_d).contiguous()
+    return sub, (sq, sk, sv, sdo), tok, qh
+
+
 # ------------------------------------------------------------------------------
 # The five workload recipes
 # ------------------------------------------------------------------------------

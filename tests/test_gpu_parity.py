@@ -85,6 +85,59 @@ def _subset_parity(w, row_ids, kv_heads):
     check_against_oracle(sub, stens, cut)
 
 
+def _group_parity(w, groups, kv_heads):
+    """Run the GPU on the whole workload at full size (the launch configuration the benchmark
+    times), then check whole groups x KV-head groups -- independent units -- element by
+    element against the oracle."""
+    from paper_2602_24082_b200 import binding as B
+    tens = w.tensors()
+    q, k, v, do = (x.cuda() for x in tens)
+    plan = B.plan_for(w, desc_on_device=True)
+    o, lse = B.pp_attn_fwd(plan, q, k, v, w.softmax_scale)
+    dq, dk, dv = B.pp_attn_bwd(plan, q, k, v, o, lse, do, w.softmax_scale)
+    torch.cuda.synchronize()
+    assert plan.status() == (0, 0)
+    sub, stens, tok, qh = W.slice_groups(w, tens, groups, kv_heads)
+    tok, qh, kh = tok.cuda(), qh.cuda(), torch.as_tensor(list(kv_heads)).cuda()
+    f64 = lambda x: x.float().cpu().numpy().astype(np.float64)
+    cut = (f64(o[tok][:, qh]), f64(lse[qh][:, tok]), f64(dq[tok][:, qh]), f64(dk[tok][:, kh]),
+           f64(dv[tok][:, kh]))
+    check_against_oracle(sub, stens, cut)
+    # everything outside the checked slice must at least be finite
+    for x in (o, lse, dq, dk, dv):
+        assert bool(torch.isfinite(x).all())
+
+
+def _smallest_groups(w, n):
+    sizes = sorted((p + sum(rs), ri, gi) for ri, row in enumerate(w.rows) for gi, (p, rs) in enumerate(row))
+    return [(ri, gi) for (_, ri, gi) in sizes[:n]]
+
+
+def test_config1_full_all_rows_one_kv_group():
+    w = W.config1()
+    _group_parity(w, [(r, 0) for r in range(8)], [5])
+
+
+def test_config2_full_size_sampled_group():
+    w = W.config2()
+    _group_parity(w, _smallest_groups(w, 1), [2])
+
+
+def test_config3_full_size_sampled_groups():
+    w = W.config3()
+    small = _smallest_groups(w, 3)
+    mid = sorted((p + sum(rs), ri, gi) for ri, row in enumerate(w.rows) for gi, (p, rs) in enumerate(row))
+    pick = small + [(mid[len(mid) // 2][1], mid[len(mid) // 2][2])]
+    _group_parity(w, pick, [6])
+
+
+@pytest.mark.parametrize("point", range(len(W.CONFIG4_POINTS)),
+                         ids=[f"rho{r}-n{n}" for r, n in W.CONFIG4_POINTS])
+def test_config4_full_size_sampled_group(point):
+    w = W.config4(point)
+    _group_parity(w, _smallest_groups(w, 1), [point % 8])
+
+
 def test_config1_subset():
     w = W.config1()
     lens = w.row_lengths()
