@@ -39,12 +39,13 @@ def get_workload(name: str, rank: int = 0):
     from paper_2602_24082_b200 import workloads as W
     if name == "config0":
         return W.config0()
+    from paper_2602_24082_b200 import multi
     if name == "config1":
-        return W.config1(seed=1 + rank)
+        return W.config1(seed=multi.rank_seed(1, rank))
     if name == "config2":
-        return W.config2(seed=2 + 10 * rank)
+        return W.config2(seed=multi.rank_seed(2, rank, 10))
     if name == "config3":
-        return W.config3(seed=3 + 10 * rank)
+        return W.config3(seed=multi.rank_seed(3, rank, 10))
     if name.startswith("config4"):
         point = int(name.split(":")[1]) if ":" in name else 0
         return W.config4(point)
@@ -191,6 +192,7 @@ def run_ours(args):
     from paper_2602_24082_b200 import binding as B
     from paper_2602_24082_b200 import workloads as W
     from paper_2602_24082_b200 import cost_model
+    from paper_2602_24082_b200 import multi
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -274,20 +276,11 @@ def run_ours(args):
     barrier()
     clocks = sampler.stop()
     B.pp_profile_enable(False)
-    total_ms = sum(ms)
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-    ms_per_step = total_ms / args.steps
     f_flops, b_flops = w.useful_flops()
-    flops_all = float(f_flops + b_flops)
-    tokens_all = float(T)
-    if world > 1:
-        t = torch.tensor([flops_all, tokens_all], device=dev, dtype=torch.float64)
-        dist.all_reduce(t)
-        flops_all, tokens_all = float(t[0].item()), float(t[1].item())
-    value = flops_all / (ms_per_step * 1e-3) / 1e12
+    # max over ranks of the timed region; sum over ranks of the work (one batch per rank)
+    total_ms, flops_all, tokens_all = multi.aggregate(sum(ms), float(f_flops + b_flops), float(T), dev)
+    ms_per_step = total_ms / args.steps
+    value = multi.whole_job_throughput(total_ms, args.steps, flops_all)
 
     if args.quick:
         if rank == 0:
@@ -310,11 +303,7 @@ def run_ours(args):
     barrier()
     e2e_ms, _ = timed(lambda: host(hq, hk, hv, hdo) and 0, max(3, min(args.steps, 10)))
     barrier()
-    e2e_total = sum(e2e_ms) / len(e2e_ms)
-    if world > 1:
-        t = torch.tensor([e2e_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_total = float(t.item())
+    e2e_total, _, _ = multi.aggregate(sum(e2e_ms) / len(e2e_ms), 0.0, 0.0, dev)
     e2e_value = flops_all / (e2e_total * 1e-3) / 1e12
 
     if rank != 0:
@@ -403,7 +392,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="config1")
@@ -412,7 +401,7 @@ def main():
                     help="timed steps only (no e2e, unpacked baseline or CPU leg): for profiler runs")
     args = ap.parse_args()
     if args.impl == "reference":
-        if args.steps == 100 and args.warmup == 5:
+        if args.steps == 200 and args.warmup == 5:
             args.steps, args.warmup = 3, 1
         run_reference(args)
     else:
