@@ -504,36 +504,46 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         const uint32_t g = gc + it;
         wait_bar(bar(kDqFull), g & 1, abort_flag, prm.header, 80);
         tc_fence_after();
-#pragma unroll 1
-        for (int c = 0; c < D / 32; ++c, ++chunk) {
-          const uint32_t buf = stg + (chunk & 1) * L::kStageBytes;
-          // the reduce issued two chunks ago must have finished reading this buffer
-          if (leader) bulk_wait_group_read<1>();
-          named_barrier_sync(1, 128);
-          uint32_t w[32];
-          tmem_ld32(lane_base + tdP + c * 32, w);
+        // Two halves of D/2 columns.  The second half is read out of tensor memory (and the
+        // dP/dQ columns handed back to the MMA warp) before any wait on the reductions issued
+        // for the first half, so the MMA pipeline never waits for TMA reads of the staging.
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          uint32_t w[D / 2];
+#pragma unroll
+          for (int c = 0; c < D / 64; ++c)
+            tmem_ld32(lane_base + tdP + half * (D / 2) + c * 32,
+                      *reinterpret_cast<uint32_t(*)[32]>(&w[c * 32]));
           tmem_wait_ld();
-          if (c == D / 32 - 1) {
+          if (half == 1) {
             tc_fence_before();
             mbar_arrive(bar(kDqDrained));
           }
           if (row >= qt.len) {  // rows past the tile's end belong to other tokens: add zero
 #pragma unroll
-            for (int i = 0; i < 32; ++i) w[i] = 0u;
+            for (int i = 0; i < D / 2; ++i) w[i] = 0u;
           }
-          const uint32_t row_addr = buf + row * 128;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const uint32_t ch = uint32_t(i) ^ uint32_t(row & 7);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + ch * 16),
-                         "r"(w[4 * i]), "r"(w[4 * i + 1]), "r"(w[4 * i + 2]), "r"(w[4 * i + 3])
-                         : "memory");
-          }
-          fence_proxy_async_smem();
-          named_barrier_sync(1, 128);
-          if (leader) {
-            tma_reduce_add_3d(&tm_dq, buf, c * 32, qt.h, qt.start);
-            bulk_commit_group();
+          for (int c = 0; c < D / 64; ++c, ++chunk) {
+            const uint32_t buf = stg + (chunk & 1) * L::kStageBytes;
+            // the reduce issued two chunks ago must have finished reading this buffer
+            if (leader) bulk_wait_group_read<1>();
+            named_barrier_sync(1, 128);
+            const uint32_t row_addr = buf + row * 128;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const uint32_t ch = uint32_t(i) ^ uint32_t(row & 7);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + ch * 16),
+                           "r"(w[c * 32 + 4 * i]), "r"(w[c * 32 + 4 * i + 1]),
+                           "r"(w[c * 32 + 4 * i + 2]), "r"(w[c * 32 + 4 * i + 3])
+                           : "memory");
+            }
+            fence_proxy_async_smem();
+            named_barrier_sync(1, 128);
+            if (leader) {
+              tma_reduce_add_3d(&tm_dq, buf, half * (D / 2) + c * 32, qt.h, qt.start);
+              bulk_commit_group();
+            }
           }
         }
       }
