@@ -317,9 +317,13 @@ def run_ours(args):
     bwd_ms = statistics.mean(x[1] for x in kern)
     bwd_tflops = b_flops / (bwd_ms * 1e-3) / 1e12
     fwd_tflops = f_flops / (fwd_ms * 1e-3) / 1e12
+    # DRAM bytes per launch of the backward main kernel from one ncu capture of this workload
+    # (profiles/fwd_bwd_kernels_config1.md); other workloads have no capture -> null
+    traffic = 1.0628e9 if args.config == "config1" else None
     roofline = {"kernel": "bwd_kernel (dS/dQ/dK/dV main)", "bound": "tensor", "achieved": bwd_tflops,
                 "peak": peak, "unit": "TFLOP/s", "frac": bwd_tflops / peak, "peak_kind": f"of {peak_kind} (burst)",
-                "traffic": None, "avg_launch_ms": bwd_ms}
+                "traffic": traffic, "traffic_unit": "bytes (dram read + write per launch)",
+                "algorithmic_flops_per_launch": float(b_flops), "avg_launch_ms": bwd_ms}
     roofline_fwd = {"kernel": "fwd_kernel", "bound": "tensor", "achieved": fwd_tflops, "peak": peak,
                     "unit": "TFLOP/s", "frac": fwd_tflops / peak, "avg_launch_ms": fwd_ms}
 
