@@ -322,6 +322,7 @@ def run_ours(args):
     traffic = 1.0628e9 if args.config == "config1" else None
     roofline = {"kernel": "bwd_kernel (dS/dQ/dK/dV main)", "bound": "tensor", "achieved": bwd_tflops,
                 "peak": peak, "unit": "TFLOP/s", "frac": bwd_tflops / peak, "peak_kind": f"of {peak_kind} (burst)",
+                "frac_of_sustained_peak": bwd_tflops / peak_sustained,
                 "traffic": traffic, "traffic_unit": "bytes (dram read + write per launch)",
                 "algorithmic_flops_per_launch": float(b_flops), "avg_launch_ms": bwd_ms}
     roofline_fwd = {"kernel": "fwd_kernel", "bound": "tensor", "achieved": fwd_tflops, "peak": peak,
