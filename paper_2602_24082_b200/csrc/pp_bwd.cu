@@ -122,7 +122,9 @@ enum BwdBar : int {
   kDqDrained,    // 128
   kDkvFull,
   kDkvFree,      // 256
-  kNumBwdBars
+  kSchedFull,    // [2]  unit ids handed from the producer warp to the other roles
+  kSchedEmpty = kSchedFull + 2,  // [2]  13 arrivals: MMA thread + 8 compute warps + 4 dQ warps
+  kNumBwdBars = kSchedEmpty + 2
 };
 
 template <int D>
@@ -132,7 +134,7 @@ struct BwdSmem {
   static constexpr int kK = 0, kV = kTileBytes, kQ = 2 * kTileBytes, kdO = 4 * kTileBytes,
                        kStg = 5 * kTileBytes, kdS = kStg + 2 * kStageBytes,
                        kStats = kdS + 128 * 128 * 2, kBars = kStats + 2 * 256 * 4;
-  static constexpr int kUsed = kBars + 8 * kNumBwdBars + 16;
+  static constexpr int kUsed = kBars + 8 * kNumBwdBars + 32;
   // The declared 1024-byte alignment of the dynamic shared memory leaves no slack to spend at
   // D = 128 (227 KB limit); the kernel checks the base and reports if it is not aligned.
   static constexpr int kTotal = kUsed + (kUsed + 1024 <= 232448 ? 1024 : 0);
@@ -143,10 +145,12 @@ struct BwdUnit {
   int kvh, nq, n_it;
 };
 
-__device__ __forceinline__ int bwd_unit_of_round(int round) {
-  const int g = gridDim.x, b = blockIdx.x;
-  return round * g + ((round & 1) ? (g - 1 - b) : b);
-}
+// Units are handed out dynamically: the producer warp draws the next index of the plan's
+// longest-work-first order from a global counter whenever the CTA is ready for more (list
+// scheduling), and passes it to the other roles through a two-entry shared-memory ring.
+// header[5] is that counter, header[7] counts finished CTAs; the last one resets both, so a
+// plan can be used by any number of launches without a memset in between.
+constexpr int kHdrBwdNext = 5, kHdrBwdDone = 7;
 
 __device__ __forceinline__ bool get_bwd_unit(const BwdParams& prm, int u, int ntiles_total,
                                              BwdUnit& un) {
@@ -222,6 +226,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       if (i == kQFullB || i == kQFullB + 1) cnt = 33;
       if (i == kPReady || i == kDsReady || i == kDkvFree) cnt = 256;
       if (i == kDqDrained) cnt = 128;
+      if (i == kSchedEmpty || i == kSchedEmpty + 1) cnt = 13;
       mbar_init(bar(i), cnt);
     }
     *abort_flag = 0;
@@ -241,12 +246,36 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   tc_fence_after();
   const uint32_t tmem = *tmem_slot_p;
   constexpr uint32_t tS = 0, tdP = 128, tdV = 256, tdK = 384;
+  volatile int* sched = reinterpret_cast<volatile int*>(gbase + L::kBars + 8 * kNumBwdBars + 16);
+  // producer warp (all lanes): draw the n-th unit of this CTA and publish it
+  auto fetch_unit = [&](uint32_t n) -> int {
+    int u = 0;
+    if (lane == 0) {
+      wait_bar(bar(kSchedEmpty + (n & 1)), ((n >> 1) & 1) ^ 1, abort_flag, prm.header, 90);
+      u = atomicAdd(&prm.header[kHdrBwdNext], 1);
+      sched[n & 1] = u;
+      mbar_arrive(bar(kSchedFull + (n & 1)));
+    }
+    return __shfl_sync(0xffffffffu, u, 0);
+  };
+  // other roles: read the n-th unit; `whole_warp` = all 32 lanes are calling
+  auto take_unit = [&](uint32_t n, bool whole_warp) -> int {
+    const bool ok = wait_bar(bar(kSchedFull + (n & 1)), (n >> 1) & 1, abort_flag, prm.header, 91);
+    const int u = ok ? sched[n & 1] : 0x7fffffff;
+    if (whole_warp) {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(kSchedEmpty + (n & 1)));
+    } else {
+      mbar_arrive(bar(kSchedEmpty + (n & 1)));
+    }
+    return u;
+  };
 
   if (warp == 0) {
     // ------------------------------------------------------------ producer
     uint32_t qc = 0, ucnt = 0;
     BwdUnit un;
-    for (int rnd = 0; get_bwd_unit(prm, bwd_unit_of_round(rnd), ntiles_total, un); ++rnd, ++ucnt) {
+    for (; get_bwd_unit(prm, fetch_unit(ucnt), ntiles_total, un); ++ucnt) {
       if (lane == 0) {
         wait_bar(bar(kKvEmpty), (ucnt & 1) ^ 1, abort_flag, prm.header, 50);
         mbar_expect_tx(bar(kKvFull), 2 * L::kTileBytes);
@@ -309,7 +338,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           mma_ss(tmem + tS, dK_k + kmajor_off(k), dq_k + kmajor_off(k), idesc, k > 0);
         mma_commit(bar(kSFullB));
       };
-      for (int rnd = 0; get_bwd_unit(prm, bwd_unit_of_round(rnd), ntiles_total, un); ++rnd, ++ucnt) {
+      for (; get_bwd_unit(prm, take_unit(ucnt, false), ntiles_total, un); ++ucnt) {
         const int ksteps = (un.tile.len + 15) >> 4;
         wait_bar(bar(kKvFull), ucnt & 1, abort_flag, prm.header, 60);
         QIter qi;
@@ -382,7 +411,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const int cb = 64 * wg;
     uint32_t gc = 0, ucnt = 0;
     BwdUnit un;
-    for (int rnd = 0; get_bwd_unit(prm, bwd_unit_of_round(rnd), ntiles_total, un); ++rnd, ++ucnt) {
+    for (; get_bwd_unit(prm, take_unit(ucnt, true), ntiles_total, un); ++ucnt) {
       const bool row_ok = row < un.tile.len;
       QIter qi;
       for (int it = 0; it < un.n_it; ++it, q_advance(qi, un.nq)) {
@@ -495,9 +524,9 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const bool leader = (warp == 10 && lane == 0);
     const uint32_t lane_base = tmem + (uint32_t(32 * (warp & 3)) << 16);
     const uint32_t stg = base + L::kStg;
-    uint32_t gc = 0, chunk = 0;
+    uint32_t gc = 0, chunk = 0, ucnt = 0;
     BwdUnit un;
-    for (int rnd = 0; get_bwd_unit(prm, bwd_unit_of_round(rnd), ntiles_total, un); ++rnd) {
+    for (; get_bwd_unit(prm, take_unit(ucnt, true), ntiles_total, un); ++ucnt) {
       QIter qi;
       for (int it = 0; it < un.n_it; ++it, q_advance(qi, un.nq)) {
         const QTile qt = q_tile_at(prm, un, qi);
@@ -555,6 +584,13 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, kBwdTmemCols);
+  if (tid == 0) {  // the last CTA to finish re-arms the unit counter for the next launch
+    __threadfence();
+    if (atomicAdd(&prm.header[kHdrBwdDone], 1) == int(gridDim.x) - 1) {
+      prm.header[kHdrBwdNext] = 0;
+      prm.header[kHdrBwdDone] = 0;
+    }
+  }
 #ifdef PP_TIMING
   if (blockIdx.x == 0 && tid == 0) g_wait_cycles[127] = (unsigned long long)(clock64() - t_kernel0);
   if (tid == 0) g_cta_cycles[blockIdx.x & 255] = (unsigned long long)(clock64() - t_kernel0);

@@ -46,6 +46,7 @@ __device__ __forceinline__ bool plan_scan_body(const PlanPtrs& p) {
     p.header[1] = 0;
     p.header[2] = 0;
     p.header[3] = p.nseg;
+    for (int i = 4; i < 8; ++i) p.header[i] = 0;  // dynamic-scheduling counters of the kernels
     if (p.row_group_off[0] != 0 || p.row_group_off[p.num_rows] != p.G)
       set_status(p.header, kStatusBadDescriptor, -1);
     if (p.grp_resp_off[0] != 0 || p.grp_resp_off[p.G] != p.N)
