@@ -46,7 +46,9 @@ enum FwdBar : int {
   kPFull = 14,
   kODone = 16,
   kOFree = 18,
-  kNumFwdBars = 20
+  kSchedFullF = 20,   // [2] unit ids handed from the producer to the other roles
+  kSchedEmptyF = 22,  // [2] 9 arrivals: MMA thread + 8 softmax warps
+  kNumFwdBars = 24
 };
 
 template <int D>
@@ -84,12 +86,11 @@ struct Unit {
   int h0, kvh, nslots, n0, n1, ntiles;
 };
 
-// Units are sorted longest first; CTA b takes unit b of round 0, the mirrored position of
-// round 1, and so on (boustrophedon), which evens out the per-CTA sums of a sorted list.
-__device__ __forceinline__ int unit_of_round(int round) {
-  const int g = gridDim.x, b = blockIdx.x;
-  return round * g + ((round & 1) ? (g - 1 - b) : b);
-}
+// Units are handed out dynamically in the plan's longest-work-first order: the producer
+// draws the next index from a global counter (header[4]) when the CTA is ready for more and
+// passes it on through a two-entry shared-memory ring; header[6] counts finished CTAs and the
+// last one resets both counters for the next launch.
+constexpr int kHdrFwdNext = 4, kHdrFwdDone = 6;
 
 __device__ __forceinline__ bool get_unit(const FwdParams& prm, int u, int ntiles_total, Unit& un) {
   const int r = prm.Hq / prm.Hkv, npairs = (r + 1) >> 1, per_tile = prm.Hkv * npairs;
@@ -133,7 +134,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   if (tid == 0) {
     for (int i = 0; i < kNumFwdBars; ++i) {
       const bool wg_count = (i >= kPFull && i < kPFull + 2) || (i >= kOFree && i < kOFree + 2);
-      mbar_init(bar(i), wg_count ? 128 : 1);
+      const bool sched_empty = (i >= kSchedEmptyF && i < kSchedEmptyF + 2);
+      mbar_init(bar(i), wg_count ? 128 : (sched_empty ? 9 : 1));
     }
     *abort_flag = 0;
     fence_mbar_init();
@@ -149,13 +151,32 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot_p;
+  volatile int* sched = reinterpret_cast<volatile int*>(gbase + L::kBars + 8 * kNumFwdBars + 16);
+  auto fetch_unit = [&](uint32_t n) -> int {  // producer thread
+    wait_bar(bar(kSchedEmptyF + (n & 1)), ((n >> 1) & 1) ^ 1, abort_flag, prm.header, 90);
+    const int u = atomicAdd(&prm.header[kHdrFwdNext], 1);
+    sched[n & 1] = u;
+    mbar_arrive(bar(kSchedFullF + (n & 1)));
+    return u;
+  };
+  auto take_unit = [&](uint32_t n, bool whole_warp) -> int {
+    const bool ok = wait_bar(bar(kSchedFullF + (n & 1)), (n >> 1) & 1, abort_flag, prm.header, 91);
+    const int u = ok ? sched[n & 1] : 0x7fffffff;
+    if (whole_warp) {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(kSchedEmptyF + (n & 1)));
+    } else {
+      mbar_arrive(bar(kSchedEmptyF + (n & 1)));
+    }
+    return u;
+  };
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       uint32_t kc = 0, vc = 0, qc[2] = {0, 0};
       Unit un;
-      for (int rnd = 0; get_unit(prm, unit_of_round(rnd), ntiles_total, un); ++rnd) {
+      for (uint32_t un_i = 0; get_unit(prm, fetch_unit(un_i), ntiles_total, un); ++un_i) {
         for (int s = 0; s < un.nslots; ++s) {
           wait_bar(bar(kQEmpty + s), (qc[s] & 1) ^ 1, abort_flag, prm.header, 20 + s);
           mbar_expect_tx(bar(kQFull + s), L::kTileBytes);
@@ -200,7 +221,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           mma_ss(tmem + s * 128, dq + kmajor_off(kk), dk + kmajor_off(kk), idesc_s, kk > 0);
         mma_commit(bar(kSFull + s));
       };
-      for (int rnd = 0; get_unit(prm, unit_of_round(rnd), ntiles_total, un); ++rnd) {
+      for (uint32_t un_i = 0; get_unit(prm, take_unit(un_i, false), ntiles_total, un); ++un_i) {
         for (int s = 0; s < un.nslots; ++s)
           wait_bar(bar(kQFull + s), uc[s] & 1, abort_flag, prm.header, 30 + s);
         KvTile kt = kv_tile_of(un.tile, 0, un.n0, un.n1);
@@ -257,7 +278,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const uint32_t tS = lane_base + s * 128, tO = lane_base + 256 + s * 128;
     uint32_t tcS = 0;
     Unit un;
-    for (int rnd = 0; get_unit(prm, unit_of_round(rnd), ntiles_total, un); ++rnd) {
+    for (uint32_t un_i = 0; get_unit(prm, take_unit(un_i, true), ntiles_total, un); ++un_i) {
       if (s >= un.nslots) continue;
       float m_used = -INFINITY, l_run = 0.f;
       for (int j = 0; j < un.ntiles; ++j) {
@@ -362,6 +383,13 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, kFwdTmemCols);
+  if (tid == 0) {  // the last CTA to finish re-arms the unit counter for the next launch
+    __threadfence();
+    if (atomicAdd(&prm.header[kHdrFwdDone], 1) == int(gridDim.x) - 1) {
+      prm.header[kHdrFwdNext] = 0;
+      prm.header[kHdrFwdDone] = 0;
+    }
+  }
 #ifdef PP_TIMING
   if (blockIdx.x == 0 && tid == 0) g_wait_cycles[127] = (unsigned long long)(clock64() - t_kernel0);
   if (tid == 0) g_cta_cycles[blockIdx.x & 255] = (unsigned long long)(clock64() - t_kernel0);
