@@ -79,7 +79,10 @@ int pp_plan_workspace_bytes(const pp_problem* problem, size_t* plan_bytes,
  * (class FULL: no masking), then its own diagonal tile (class DIAG: causal masking) --
  * while tiles of sibling responses are never listed (class SKIP is implicit).  The same
  * tiles, read as key tiles, carry the contiguous query range [start, vis_end) that sees
- * them, for the backward pass.  Tiles are ordered longest-work-first for both passes.
+ * them, for the backward pass.  Tiles are ordered longest-work-first for the forward pass;
+ * the backward pass processes (tile, KV head) units group by group (largest group first,
+ * longest tile first inside a group) so that concurrently running units share Q / dO in L2.
+ * Both kernels draw units dynamically, so the order is a priority list, not an assignment.
  * d_workspace must stay alive and untouched while the plan is used.  The plan is
  * immutable and can be reused by any number of pp_attn_fwd / pp_attn_bwd calls whose
  * tensors have the shapes stated in `problem`.
@@ -101,6 +104,10 @@ int pp_destroy_plan(pp_plan* plan);
  * per token j, the first query index that can NOT see key j.  Any pointer may be NULL.
  * *num_tiles receives the tile count; arrays must hold pp_plan_max_tiles entries. */
 int pp_plan_max_tiles(const pp_plan* plan);
+/* Backward processing order: max_tiles * Hkv records (kv_head << 24) | tile, of which the
+ * first num_tiles * Hkv are valid.  Units of one group are adjacent (they stream the same
+ * Q / dO tiles through L2), groups with the most work first.  Synchronises `stream`. */
+int pp_plan_read_bwd_units(const pp_plan* plan, pp_stream_t stream, int32_t* units);
 int pp_plan_read(const pp_plan* plan, pp_stream_t stream, int32_t* num_tiles, int32_t* tiles,
                  int32_t* fwd_order, int32_t* bwd_order, int32_t* key_end);
 

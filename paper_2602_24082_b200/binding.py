@@ -24,7 +24,7 @@ EXPORTS = ["pp_plan_workspace_bytes", "pp_build_plan", "pp_plan_status", "pp_des
            "pp_plan_max_tiles", "pp_plan_read", "pp_attn_fwd", "pp_attn_bwd",
            "pp_last_launch_count", "pp_error_string", "pp_step_host_arena_bytes",
            "pp_attn_step_host", "pp_profile_enable", "pp_profile_read",
-           "pp_attn_bwd_noalloc", "pp_attn_bwd_noalloc_max_bytes"]
+           "pp_attn_bwd_noalloc", "pp_attn_bwd_noalloc_max_bytes", "pp_plan_read_bwd_units"]
 
 
 class PPError(RuntimeError):
@@ -65,6 +65,7 @@ def lib() -> ctypes.CDLL:
         L.pp_plan_status.argtypes = [vp, vp, vp, vp]
         L.pp_destroy_plan.argtypes = [vp]
         L.pp_plan_max_tiles.argtypes = [vp]
+        L.pp_plan_read_bwd_units.argtypes = [vp, vp, vp]
         L.pp_plan_read.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         L.pp_attn_fwd.argtypes = [vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, sz, vp]
         L.pp_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, sz, vp]
@@ -124,6 +125,16 @@ class Plan:
         _check(lib().pp_plan_read(self.handle, _stream(), ctypes.byref(n), tiles.ctypes.data,
                                   fo.ctypes.data, bo.ctypes.data, ke.ctypes.data), "pp_plan_read")
         return tiles[:n.value], fo[:n.value], bo[:n.value], ke
+
+    def read_bwd_units(self, num_tiles: int) -> np.ndarray:
+        """The backward processing order as (kv_head, tile) rows."""
+        mt = lib().pp_plan_max_tiles(self.handle)
+        hkv = self.problem.num_kv_heads
+        raw = np.zeros(mt * hkv, dtype=np.int32)
+        _check(lib().pp_plan_read_bwd_units(self.handle, _stream(), raw.ctypes.data),
+               "pp_plan_read_bwd_units")
+        raw = raw[:num_tiles * hkv]
+        return np.stack([raw >> 24, raw & 0xffffff], axis=1)
 
     def __del__(self):
         try:

@@ -19,6 +19,9 @@ int check_problem_shape(const pp_problem* p) {
   if (p->num_q_heads < 1 || p->num_kv_heads < 1 || p->num_q_heads % p->num_kv_heads != 0)
     return PP_ERR_INVALID_ARG;
   if (p->head_dim != 64 && p->head_dim != 128) return PP_ERR_UNSUPPORTED;
+  // unit records pack (kv head << 24) | tile
+  if (p->num_kv_heads > 127 || p->total_tokens / 128 + p->num_groups + p->num_responses >= (1 << 24))
+    return PP_ERR_UNSUPPORTED;
   return PP_OK;
 }
 
@@ -138,6 +141,17 @@ int pp_destroy_plan(pp_plan* plan) {
 }
 
 int pp_plan_max_tiles(const pp_plan* plan) { return plan ? plan->max_tiles : PP_ERR_INVALID_ARG; }
+
+int pp_plan_read_bwd_units(const pp_plan* plan, pp_stream_t stream, int32_t* units) {
+  if (!plan || !units) return PP_ERR_INVALID_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  const size_t n = size_t(plan->max_tiles) * plan->prob.num_kv_heads;
+  if (cudaMemcpyAsync(units, plan->ws + plan->lay.bwd_units, n * 4, cudaMemcpyDeviceToHost, s) !=
+          cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess)
+    return PP_ERR_CUDA;
+  return PP_OK;
+}
 
 int pp_plan_read(const pp_plan* plan, pp_stream_t stream, int32_t* num_tiles, int32_t* tiles,
                  int32_t* fwd_order, int32_t* bwd_order, int32_t* key_end) {

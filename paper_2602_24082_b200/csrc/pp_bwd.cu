@@ -154,10 +154,10 @@ constexpr int kHdrBwdNext = 5, kHdrBwdDone = 7;
 
 __device__ __forceinline__ bool get_bwd_unit(const BwdParams& prm, int u, int ntiles_total,
                                              BwdUnit& un) {
-  const int ord = u / prm.Hkv;
-  if (ord >= ntiles_total) return false;
-  un.kvh = u - ord * prm.Hkv;
-  un.tile = prm.tiles[prm.order[ord]];
+  if (u < 0 || u >= ntiles_total * prm.Hkv) return false;
+  const int packed = prm.order[u];  // (kv head << 24) | tile
+  un.kvh = packed >> 24;
+  un.tile = prm.tiles[packed & 0xffffff];
   const int full_len = un.tile.vis_end - (un.tile.start + un.tile.len);
   un.nq = 1 + (full_len + kTile - 1) / kTile;
   un.n_it = un.nq * (prm.Hq / prm.Hkv);
@@ -677,7 +677,7 @@ cudaError_t launch_bwd(const pp_plan* plan, const void* q, const void* k, const 
   BwdParams prm;
   prm.header = reinterpret_cast<int32_t*>(plan->ws + plan->lay.header);
   prm.tiles = reinterpret_cast<const Tile*>(plan->ws + plan->lay.tiles);
-  prm.order = reinterpret_cast<const int32_t*>(plan->ws + plan->lay.bwd_order);
+  prm.order = reinterpret_cast<const int32_t*>(plan->ws + plan->lay.bwd_units);
   prm.delta = reinterpret_cast<float*>(sc + sl.delta);
   prm.lse2 = reinterpret_cast<float*>(sc + sl.lse2);
   prm.dq_acc = reinterpret_cast<float*>(sc + sl.dq_acc);

@@ -41,6 +41,9 @@ struct PlanLayout {
   size_t tiles;      // Tile[max_tiles]
   size_t fwd_order;  // int32[max_tiles]
   size_t bwd_order;  // int32[max_tiles]
+  size_t tile_gwork; // int32[max_tiles]  backward work of the tile's whole group
+  size_t tile_sgroup; // int32[max_tiles] super-group (block of consecutive groups) of the tile
+  size_t bwd_units;  // int32[max_tiles * Hkv]  (kv head << 24) | tile, in processing order
   size_t key_end;    // int32[T]
   size_t total;
 };
@@ -80,6 +83,9 @@ inline PlanLayout plan_layout(const pp_problem& p) {
   l.tiles = off;     off = align_up(off + sizeof(Tile) * size_t(mt), 256);
   l.fwd_order = off; off = align_up(off + sizeof(int32_t) * size_t(mt), 256);
   l.bwd_order = off; off = align_up(off + sizeof(int32_t) * size_t(mt), 256);
+  l.tile_gwork = off; off = align_up(off + sizeof(int32_t) * size_t(mt), 256);
+  l.tile_sgroup = off; off = align_up(off + sizeof(int32_t) * size_t(mt), 256);
+  l.bwd_units = off; off = align_up(off + sizeof(int32_t) * size_t(mt) * size_t(p.num_kv_heads), 256);
   l.key_end = off;   off = align_up(off + sizeof(int32_t) * size_t(p.total_tokens), 256);
   l.total = off;
   return l;

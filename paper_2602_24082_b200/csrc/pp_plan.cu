@@ -22,6 +22,10 @@ struct PlanPtrs {
   Tile* tiles;
   int32_t* fwd_order;
   int32_t* bwd_order;
+  int32_t* tile_gwork;
+  int32_t* tile_sgroup;
+  int32_t* bwd_units;
+  int Hkv;
   int32_t* key_end;
   int num_rows, G, N, T, nseg, max_tiles;
 };
@@ -211,6 +215,69 @@ __global__ void plan_order_kernel(PlanPtrs p) {
   if (t < n) plan_order_body(p, t, n);
 }
 
+// Backward processing order, built for L2 reuse and balance.  Key tiles of one group stream
+// the same Q / dO tiles, so groups are taken in order of decreasing work and consecutive
+// groups are merged into super-groups of about kSuperGroupUnits units (cut from the end of
+// the list, so the last block is a full one); inside a super-group
+// units are ordered longest first (all KV heads of a tile adjacent).  Small problems collapse
+// into one super-group, i.e. a plain longest-first list; large ones keep the working set of the
+// concurrently running units near one group's Q / dO.  Dynamic scheduling in the kernel does
+// the balancing.  A tile's group is identified by the start of its prompt range (kv0_start).
+constexpr int kSuperGroupUnits = 600;
+
+__device__ __forceinline__ void plan_gwork_body(const PlanPtrs& p, int t, int n) {
+  const int gs = p.tiles[t].kv0_start;
+  int gw = 0;
+  for (int u = 0; u < n; ++u) {
+    Tile o = p.tiles[u];
+    gw += (o.kv0_start == gs) ? bwd_work(o) : 0;
+  }
+  p.tile_gwork[t] = gw;
+}
+
+__device__ __forceinline__ void plan_sgroup_body(const PlanPtrs& p, int t, int n) {
+  const int gs = p.tiles[t].kv0_start, gw = p.tile_gwork[t];
+  int rest = 0;  // tiles of this group and of the groups that come later
+  for (int u = 0; u < n; ++u) {
+    const int ogs = p.tiles[u].kv0_start, ow = p.tile_gwork[u];
+    rest += (ogs == gs) || (ow < gw) || (ow == gw && ogs > gs);
+  }
+  // counted from the END of the list, so the last block is never a small leftover whose
+  // long units would start late: blocks are processed in decreasing index
+  p.tile_sgroup[t] = (p.Hkv * rest - 1) / kSuperGroupUnits;
+}
+
+__device__ __forceinline__ void plan_units_body(const PlanPtrs& p, int t, int n) {
+  const int sg = p.tile_sgroup[t], wb = bwd_work(p.tiles[t]);
+  int pos = 0;
+  for (int u = 0; u < n; ++u) {
+    const int osg = p.tile_sgroup[u], ob = bwd_work(p.tiles[u]);
+    pos += (osg > sg) || (osg == sg && ((ob > wb) || (ob == wb && u < t)));
+  }
+  for (int kvh = 0; kvh < p.Hkv; ++kvh) p.bwd_units[p.Hkv * pos + kvh] = (kvh << 24) | t;
+}
+
+__global__ void plan_gwork_kernel(PlanPtrs p) {
+  if (p.header[0] != kStatusOk) return;
+  const int n = p.header[2];
+  int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t < n) plan_gwork_body(p, t, n);
+}
+
+__global__ void plan_sgroup_kernel(PlanPtrs p) {
+  if (p.header[0] != kStatusOk) return;
+  const int n = p.header[2];
+  int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t < n) plan_sgroup_body(p, t, n);
+}
+
+__global__ void plan_units_kernel(PlanPtrs p) {
+  if (p.header[0] != kStatusOk) return;
+  const int n = p.header[2];
+  int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t < n) plan_units_body(p, t, n);
+}
+
 // The whole plan in one block: used when the problem is small enough that one block's
 // latency beats four dependent launches (every stage only needs block-level ordering).
 __global__ void __launch_bounds__(1024) plan_fused_kernel(PlanPtrs p) {
@@ -219,7 +286,14 @@ __global__ void __launch_bounds__(1024) plan_fused_kernel(PlanPtrs p) {
   for (int t = threadIdx.x; t < n; t += blockDim.x) plan_tile_body(p, t);
   for (int j = threadIdx.x; j < p.T; j += blockDim.x) plan_key_end_body(p, j);
   __syncthreads();
-  for (int t = threadIdx.x; t < n; t += blockDim.x) plan_order_body(p, t, n);
+  for (int t = threadIdx.x; t < n; t += blockDim.x) {
+    plan_order_body(p, t, n);
+    plan_gwork_body(p, t, n);
+  }
+  __syncthreads();
+  for (int t = threadIdx.x; t < n; t += blockDim.x) plan_sgroup_body(p, t, n);
+  __syncthreads();
+  for (int t = threadIdx.x; t < n; t += blockDim.x) plan_units_body(p, t, n);
 }
 
 }  // namespace
@@ -268,6 +342,10 @@ cudaError_t launch_plan(const pp_plan* plan, cudaStream_t stream, int* launches)
   p.tiles = reinterpret_cast<Tile*>(ws + l.tiles);
   p.fwd_order = reinterpret_cast<int32_t*>(ws + l.fwd_order);
   p.bwd_order = reinterpret_cast<int32_t*>(ws + l.bwd_order);
+  p.tile_gwork = reinterpret_cast<int32_t*>(ws + l.tile_gwork);
+  p.tile_sgroup = reinterpret_cast<int32_t*>(ws + l.tile_sgroup);
+  p.bwd_units = reinterpret_cast<int32_t*>(ws + l.bwd_units);
+  p.Hkv = plan->prob.num_kv_heads;
   p.key_end = reinterpret_cast<int32_t*>(ws + l.key_end);
   p.num_rows = plan->prob.num_rows;
   p.G = plan->prob.num_groups;
@@ -286,7 +364,10 @@ cudaError_t launch_plan(const pp_plan* plan, cudaStream_t stream, int* launches)
   plan_tiles_kernel<<<(mt + 255) / 256, 256, 0, stream>>>(p);
   plan_key_end_kernel<<<(p.T + 255) / 256, 256, 0, stream>>>(p);
   plan_order_kernel<<<(mt + 127) / 128, 128, 0, stream>>>(p);
-  if (launches) *launches = 4;
+  plan_gwork_kernel<<<(mt + 127) / 128, 128, 0, stream>>>(p);
+  plan_sgroup_kernel<<<(mt + 127) / 128, 128, 0, stream>>>(p);
+  plan_units_kernel<<<(mt + 127) / 128, 128, 0, stream>>>(p);
+  if (launches) *launches = 7;
   return cudaGetLastError();
 }
 

@@ -73,6 +73,32 @@ def test_plan_matches_dense_mask(w, desc_on_device):
     assert (np.diff(bw[bwd_order]) <= 0).all()
 
 
+@pytest.mark.parametrize("w", CASES + [W.config4(3)], ids=lambda w: w.name)
+def test_backward_units_order(w):
+    """Every (tile, KV head) appears exactly once; groups are taken in order of decreasing
+    backward work and merged into super-groups of about 600 units; inside a super-group units
+    come longest first with all KV heads of a tile adjacent."""
+    from paper_2602_24082_b200 import binding as B
+    plan = B.plan_for(w, desc_on_device=True)
+    tiles, _, _, _ = plan.read()
+    n, hkv = len(tiles), w.num_kv_heads
+    units = plan.read_bwd_units(n)
+    assert units.shape == (n * hkv, 2)
+    assert sorted(map(tuple, units.tolist())) == [(h, t) for h in range(hkv) for t in range(n)]
+    work = 1 + (tiles[:, 6] - tiles[:, 0] - tiles[:, 1] + 127) // 128
+    grp = tiles[:, 2]                      # start of the group's prompt = group identity
+    gwork = {int(g): int(work[grp == g].sum()) for g in np.unique(grp)}
+    ranked = sorted(gwork, key=lambda g: (-gwork[g], g))
+    sgroup, rest = {}, n
+    for g in ranked:
+        sgroup[g] = (hkv * rest - 1) // 600     # blocks are cut from the end of the list
+        rest -= int((grp == g).sum())
+    expect = sorted(range(n), key=lambda t: (-sgroup[int(grp[t])], -int(work[t]), t))
+    assert units[:, 1].reshape(n, hkv)[:, 0].tolist() == expect
+    assert (units[:, 0].reshape(n, hkv) == np.arange(hkv)).all()
+    assert (units[:, 1].reshape(n, hkv) == units[:, 1].reshape(n, hkv)[:, :1]).all()
+
+
 def test_device_side_validation_reports_status():
     from paper_2602_24082_b200 import binding as B
     w = W.Workload("bad", [[(5, (2, 4))], [(3, (1, 2))]], 2, 1, 64, seed=0)
