@@ -361,6 +361,22 @@ def run_ours(args):
             "attention_cost_ratio": statistics.mean(cost_model.attention_cost_ratio(p, rs) for p, rs in grp),
             "memory_ratio": statistics.mean(cost_model.memory_ratio(p, rs) for p, rs in grp)}
 
+    # ---- next row of the path: packed position ids + rotary embedding on Q/K (HBM-bound)
+    if world == 1:
+        rplan = plan_holder["plan"]
+        rq, rk = q.clone(), k.clone()
+        for _ in range(3):
+            B.pp_rope_qk(rplan, rq, rk, 500000.0)
+        rms, _ = timed(lambda: (B.pp_rope_qk(rplan, rq, rk, 500000.0), 0)[1], 10)
+        rbytes = 2.0 * 2.0 * T * (Hq + Hkv) * D
+        hbm = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["hbm_gbs"] \
+            if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else 6650.0
+        gbs = rbytes / (statistics.median(rms) * 1e-3) / 1e9
+        extra["rope_qk"] = {"ms": statistics.median(rms), "bytes": rbytes,
+                            "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s",
+                                         "frac": gbs / hbm}}
+        del rq, rk
+
     # ---- the CPU oracle beside it (rank 0, N = 1 only), on a bounded sample
     cpu = None
     if world == 1 and not args.no_cpu_baseline:

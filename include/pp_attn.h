@@ -132,6 +132,19 @@ int pp_attn_bwd(const pp_plan* plan, const void* q, const void* k, const void* v
                 void* d_v, void* d_scratch, size_t scratch_bytes, pp_stream_t stream);
 
 /*
+ * The step right before attention (Sec. 3.2: "position IDs help positional embeddings retain
+ * their original positions").  pp_position_ids writes, per token, the position it would have
+ * in its own unpacked sequence (x, y^k): index inside the prompt for prompt tokens, P + index
+ * inside the response for response tokens -- positions restart after the prompt for every
+ * response.  pp_rope_qk applies the rotary embedding (rotate-half form, angle = position *
+ * rope_base^(-2i/D)) with those positions to Q [T][Hq][D] and K [T][Hkv][D] in place (bf16
+ * device pointers); V is untouched.  Both need only the plan (any plan built for the same
+ * descriptors) and run on `stream`.  position_ids: int32 device pointer, [T].
+ */
+int pp_position_ids(const pp_plan* plan, int32_t* position_ids, pp_stream_t stream);
+int pp_rope_qk(const pp_plan* plan, void* q, void* k, float rope_base, pp_stream_t stream);
+
+/*
  * pp_attn_bwd for callers that cannot allocate device memory.  (The paper has no counterpart:
  * this is a packaging variant of the backward above, not a different computation.)
  *

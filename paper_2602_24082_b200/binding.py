@@ -24,7 +24,8 @@ EXPORTS = ["pp_plan_workspace_bytes", "pp_build_plan", "pp_plan_status", "pp_des
            "pp_plan_max_tiles", "pp_plan_read", "pp_attn_fwd", "pp_attn_bwd",
            "pp_last_launch_count", "pp_error_string", "pp_step_host_arena_bytes",
            "pp_attn_step_host", "pp_profile_enable", "pp_profile_read",
-           "pp_attn_bwd_noalloc", "pp_attn_bwd_noalloc_max_bytes", "pp_plan_read_bwd_units"]
+           "pp_attn_bwd_noalloc", "pp_attn_bwd_noalloc_max_bytes", "pp_plan_read_bwd_units",
+           "pp_position_ids", "pp_rope_qk"]
 
 
 class PPError(RuntimeError):
@@ -73,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.pp_attn_step_host.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp, sz, vp]
         L.pp_attn_bwd_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
         L.pp_attn_bwd_noalloc_max_bytes.argtypes = [vp]
+        L.pp_position_ids.argtypes = [vp, vp, vp]
+        L.pp_rope_qk.argtypes = [vp, vp, vp, ctypes.c_float, vp]
         L.pp_profile_enable.argtypes = [ctypes.c_int]
         L.pp_profile_read.argtypes = [vp, vp]
         _lib = L
@@ -241,6 +244,27 @@ def pp_attn_bwd(plan: Plan, q, k, v, o, lse, d_o, softmax_scale: float, d_q=None
                                  d_q.data_ptr(), d_k.data_ptr(), d_v.data_ptr(), scratch.data_ptr(),
                                  scratch.numel(), _stream()), "pp_attn_bwd")
     return d_q, d_k, d_v
+
+
+def pp_position_ids(plan: Plan, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Packed position ids [T] int32: positions restart after the prompt for every response."""
+    if out is None:
+        out = torch.empty(plan.total_tokens, dtype=torch.int32, device=plan.workspace.device)
+    _chk(out, (plan.total_tokens,), torch.int32, "position_ids")
+    with torch.cuda.device(out.device):
+        _check(lib().pp_position_ids(plan.handle, out.data_ptr(), _stream()), "pp_position_ids")
+    return out
+
+
+def pp_rope_qk(plan: Plan, q: torch.Tensor, k: torch.Tensor, rope_base: float = 10000.0):
+    """Rotary embedding with the packed positions, in place on q [T,Hq,D] and k [T,Hkv,D]."""
+    p = plan.problem
+    _chk(q, (p.total_tokens, p.num_q_heads, p.head_dim), torch.bfloat16, "q")
+    _chk(k, (p.total_tokens, p.num_kv_heads, p.head_dim), torch.bfloat16, "k")
+    with torch.cuda.device(q.device):
+        _check(lib().pp_rope_qk(plan.handle, q.data_ptr(), k.data_ptr(), float(rope_base), _stream()),
+               "pp_rope_qk")
+    return q, k
 
 
 def pp_attn_bwd_noalloc_max_bytes() -> int:

@@ -234,6 +234,27 @@ int pp_attn_bwd_noalloc(const pp_plan* plan, const void* q, const void* k, const
   return e == cudaSuccess ? PP_OK : (e == cudaErrorNotSupported ? PP_ERR_UNSUPPORTED : PP_ERR_CUDA);
 }
 
+int pp_position_ids(const pp_plan* plan, int32_t* position_ids, pp_stream_t stream) {
+  g_last_launches = 0;
+  if (!plan || !position_ids) return PP_ERR_INVALID_ARG;
+  if (pp::launch_position_ids(plan, position_ids, reinterpret_cast<cudaStream_t>(stream)) !=
+      cudaSuccess)
+    return PP_ERR_CUDA;
+  g_last_launches = 1;
+  return PP_OK;
+}
+
+int pp_rope_qk(const pp_plan* plan, void* q, void* k, float rope_base, pp_stream_t stream) {
+  g_last_launches = 0;
+  if (!plan || !q || !k) return PP_ERR_INVALID_ARG;
+  if (!(rope_base > 1.f) || rope_base > 1e12f) return PP_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k)) return PP_ERR_ALIGNMENT;
+  if (pp::launch_rope(plan, q, k, rope_base, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return PP_ERR_CUDA;
+  g_last_launches = 1;
+  return PP_OK;
+}
+
 int pp_last_launch_count(void) { return g_last_launches; }
 
 int pp_step_host_arena_bytes(const pp_problem* problem, size_t* arena_bytes) {

@@ -149,4 +149,7 @@ cudaError_t launch_bwd_static(const pp_plan* plan, const void* q, const void* k,
                               const void* o, const float* lse, const void* d_o, float scale,
                               void* dq, void* dk, void* dv, cudaStream_t stream, int* launches);
 
+cudaError_t launch_position_ids(const pp_plan* plan, int32_t* pos, cudaStream_t stream);
+cudaError_t launch_rope(const pp_plan* plan, void* q, void* k, float base, cudaStream_t stream);
+
 }  // namespace pp
