@@ -376,6 +376,18 @@ def run_ours(args):
                             "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s",
                                          "frac": gbs / hbm}}
         del rq, rk
+        # ---- next row: loss-side consumer (per-response log-probs + pairwise preference loss)
+        tl = -torch.rand(T, device=dev) * 3
+        tr = -torch.rand(T, device=dev) * 3
+        for _ in range(3):
+            B.pp_preference_loss(rplan, tl, tr, 0.1)
+        lms, _ = timed(lambda: (B.pp_preference_loss(rplan, tl, tr, 0.1), 0)[1], 10)
+        lbytes = 12.0 * T
+        extra["preference_loss"] = {"ms": statistics.median(lms), "bytes": lbytes,
+                                    "note": "latency-bound: one warp per group, 12 bytes per token",
+                                    "roofline": {"bound": "hbm", "achieved": lbytes / (statistics.median(lms) * 1e-3) / 1e9,
+                                                 "peak": hbm, "unit": "GB/s",
+                                                 "frac": lbytes / (statistics.median(lms) * 1e-3) / 1e9 / hbm}}
 
     # ---- the CPU oracle beside it (rank 0, N = 1 only), on a bounded sample
     cpu = None

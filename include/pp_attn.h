@@ -145,6 +145,20 @@ int pp_position_ids(const pp_plan* plan, int32_t* position_ids, pp_stream_t stre
 int pp_rope_qk(const pp_plan* plan, void* q, void* k, float rope_base, pp_stream_t stream);
 
 /*
+ * The step right after the model forward (Sec. 2.1): splits the packed rows back into their
+ * responses and evaluates the preference loss.  token_logp [T] (fp32, device) holds the
+ * log-probability of each token under the policy; prompt entries are ignored.  Per response
+ * k: resp_logp = sum of its tokens' log-probs; resp_reward = beta * (resp_logp - the same sum
+ * of ref_token_logp), or beta * resp_logp when ref_token_logp is NULL.  Responses are ranked as
+ * in Sec. 3.1 (response a preferred over b for a > b); grp_loss[g] = mean over the pairs a > b
+ * of -log sigmoid(r_a - r_b) (0 for a single-response group).  d_token_logp [T] (may be NULL)
+ * receives d(sum_g grp_loss[g]) / d token_logp.  resp_logp, resp_reward: [N]; grp_loss: [G].
+ */
+int pp_preference_loss(const pp_plan* plan, const float* token_logp, const float* ref_token_logp,
+                       float beta, float* resp_logp, float* resp_reward, float* grp_loss,
+                       float* d_token_logp, pp_stream_t stream);
+
+/*
  * pp_attn_bwd for callers that cannot allocate device memory.  (The paper has no counterpart:
  * this is a packaging variant of the backward above, not a different computation.)
  *

@@ -25,7 +25,7 @@ EXPORTS = ["pp_plan_workspace_bytes", "pp_build_plan", "pp_plan_status", "pp_des
            "pp_last_launch_count", "pp_error_string", "pp_step_host_arena_bytes",
            "pp_attn_step_host", "pp_profile_enable", "pp_profile_read",
            "pp_attn_bwd_noalloc", "pp_attn_bwd_noalloc_max_bytes", "pp_plan_read_bwd_units",
-           "pp_position_ids", "pp_rope_qk"]
+           "pp_position_ids", "pp_rope_qk", "pp_preference_loss"]
 
 
 class PPError(RuntimeError):
@@ -76,6 +76,7 @@ def lib() -> ctypes.CDLL:
         L.pp_attn_bwd_noalloc_max_bytes.argtypes = [vp]
         L.pp_position_ids.argtypes = [vp, vp, vp]
         L.pp_rope_qk.argtypes = [vp, vp, vp, ctypes.c_float, vp]
+        L.pp_preference_loss.argtypes = [vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp]
         L.pp_profile_enable.argtypes = [ctypes.c_int]
         L.pp_profile_read.argtypes = [vp, vp]
         _lib = L
@@ -265,6 +266,28 @@ def pp_rope_qk(plan: Plan, q: torch.Tensor, k: torch.Tensor, rope_base: float = 
         _check(lib().pp_rope_qk(plan.handle, q.data_ptr(), k.data_ptr(), float(rope_base), _stream()),
                "pp_rope_qk")
     return q, k
+
+
+def pp_preference_loss(plan: Plan, token_logp: torch.Tensor, ref_token_logp: Optional[torch.Tensor],
+                       beta: float, want_grad: bool = True):
+    """Returns (resp_logp [N], resp_reward [N], grp_loss [G], d_token_logp [T] or None)."""
+    p = plan.problem
+    T, N, G = p.total_tokens, p.num_responses, p.num_groups
+    _chk(token_logp, (T,), torch.float32, "token_logp")
+    if ref_token_logp is not None:
+        _chk(ref_token_logp, (T,), torch.float32, "ref_token_logp")
+    dev = token_logp.device
+    resp_logp = torch.empty(N, dtype=torch.float32, device=dev)
+    resp_reward = torch.empty(N, dtype=torch.float32, device=dev)
+    grp_loss = torch.empty(G, dtype=torch.float32, device=dev)
+    grad = torch.empty(T, dtype=torch.float32, device=dev) if want_grad else None
+    with torch.cuda.device(dev):
+        _check(lib().pp_preference_loss(plan.handle, token_logp.data_ptr(),
+                                        ref_token_logp.data_ptr() if ref_token_logp is not None else None,
+                                        float(beta), resp_logp.data_ptr(), resp_reward.data_ptr(),
+                                        grp_loss.data_ptr(), grad.data_ptr() if want_grad else None,
+                                        _stream()), "pp_preference_loss")
+    return resp_logp, resp_reward, grp_loss, grad
 
 
 def pp_attn_bwd_noalloc_max_bytes() -> int:

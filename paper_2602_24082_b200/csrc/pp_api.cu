@@ -255,6 +255,20 @@ int pp_rope_qk(const pp_plan* plan, void* q, void* k, float rope_base, pp_stream
   return PP_OK;
 }
 
+int pp_preference_loss(const pp_plan* plan, const float* token_logp, const float* ref_token_logp,
+                       float beta, float* resp_logp, float* resp_reward, float* grp_loss,
+                       float* d_token_logp, pp_stream_t stream) {
+  g_last_launches = 0;
+  if (!plan || !token_logp || !resp_logp || !resp_reward || !grp_loss) return PP_ERR_INVALID_ARG;
+  if (!(beta > 0.f) || beta > 1e30f) return PP_ERR_INVALID_ARG;
+  if (pp::launch_preference_loss(plan, token_logp, ref_token_logp, beta, resp_logp, resp_reward,
+                                 grp_loss, d_token_logp,
+                                 reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return PP_ERR_CUDA;
+  g_last_launches = 1;
+  return PP_OK;
+}
+
 int pp_last_launch_count(void) { return g_last_launches; }
 
 int pp_step_host_arena_bytes(const pp_problem* problem, size_t* arena_bytes) {

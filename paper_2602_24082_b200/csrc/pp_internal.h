@@ -152,4 +152,8 @@ cudaError_t launch_bwd_static(const pp_plan* plan, const void* q, const void* k,
 cudaError_t launch_position_ids(const pp_plan* plan, int32_t* pos, cudaStream_t stream);
 cudaError_t launch_rope(const pp_plan* plan, void* q, void* k, float base, cudaStream_t stream);
 
+cudaError_t launch_preference_loss(const pp_plan* plan, const float* logp, const float* ref,
+                                   float beta, float* resp_logp, float* resp_reward,
+                                   float* grp_loss, float* d_logp, cudaStream_t stream);
+
 }  // namespace pp
