@@ -185,22 +185,32 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                         un.tile.start, bar(kQFull + s));
           ++qc[s];
         }
-        for (int j = 0; j < un.ntiles; ++j) {
+        // K runs one tile ahead of V: K(j+1) only needs QK(j-1) to be done, V(j) needs PV(j-2),
+        // so a V load waiting for its stage must not hold back the next K load.
+        auto load_k = [&](int j) {
           const KvTile kt = kv_tile_of(un.tile, j, un.n0, un.n1);
-          uint32_t st = kc & 1;
+          const uint32_t st = kc & 1;
           wait_bar(bar(kKEmpty + st), ((kc >> 1) & 1) ^ 1, abort_flag, prm.header, 22);
           mbar_expect_tx(bar(kKFull + st), L::kTileBytes);
           for (int b = 0; b < D / 64; ++b)
             tma_load_3d(sK + st * L::kTileBytes + b * kBoxBytes, &tm_k, b * 64, un.kvh, kt.start,
                         bar(kKFull + st));
           ++kc;
-          st = vc & 1;
+        };
+        auto load_v = [&](int j) {
+          const KvTile kt = kv_tile_of(un.tile, j, un.n0, un.n1);
+          const uint32_t st = vc & 1;
           wait_bar(bar(kVEmpty + st), ((vc >> 1) & 1) ^ 1, abort_flag, prm.header, 23);
           mbar_expect_tx(bar(kVFull + st), L::kTileBytes);
           for (int b = 0; b < D / 64; ++b)
             tma_load_3d(sV + st * L::kTileBytes + b * kBoxBytes, &tm_v, b * 64, un.kvh, kt.start,
                         bar(kVFull + st));
           ++vc;
+        };
+        load_k(0);
+        for (int j = 0; j < un.ntiles; ++j) {
+          if (j + 1 < un.ntiles) load_k(j + 1);
+          load_v(j);
         }
       }
     }
