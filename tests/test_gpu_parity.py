@@ -138,6 +138,20 @@ def test_config4_full_size_sampled_group(point):
     _group_parity(w, _smallest_groups(w, 1), [point % 8])
 
 
+def test_many_tiny_groups_multi_kernel_plan():
+    """More than 2048 tiles: the plan is built by the multi-kernel path instead of the fused
+    single-block kernel; segments of 1..9 tokens, several rows."""
+    rng = np.random.default_rng(5)
+    rows = []
+    for _ in range(3):
+        rows.append([(int(rng.integers(1, 10)), tuple(int(x) for x in rng.integers(1, 10, size=int(rng.integers(1, 4)))))
+                     for _ in range(420)])
+    w = W.Workload("tiny-groups", rows, 2, 1, 64, seed=77)
+    assert sum(len(rs) + 1 for row in rows for _, rs in row) > 2048
+    tens = w.tensors()
+    check_against_oracle(w, tens, _run_gpu(w, tens, desc_on_device=True))
+
+
 def test_config1_subset():
     w = W.config1()
     lens = w.row_lengths()

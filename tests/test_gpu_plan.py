@@ -99,6 +99,35 @@ def test_backward_units_order(w):
     assert (units[:, 1].reshape(n, hkv) == units[:, 1].reshape(n, hkv)[:, :1]).all()
 
 
+def test_multi_kernel_plan_path_matches_fused_semantics():
+    """> 2048 tiles forces the multi-kernel plan path; its tiles / orders obey the same
+    rules (checked through the same dense-mask comparison on a prefix of the tokens)."""
+    from paper_2602_24082_b200 import binding as B
+    rows = [[(3 + (i % 5), (1 + (i % 3), 2)) for i in range(1100)]]
+    w = W.Workload("many", rows, 2, 2, 64, seed=1)
+    plan = B.plan_for(w, desc_on_device=True)
+    assert plan.status() == (0, 0)
+    tiles, fwd_order, bwd_order, key_end = plan.read()
+    n = len(tiles)
+    assert n == 3 * 1100 and n > 2048
+    assert sorted(fwd_order.tolist()) == list(range(n)) and sorted(bwd_order.tolist()) == list(range(n))
+    segs = w.segments()
+    assert [int(t[0]) for t in tiles] == [s[0] for s in segs] and [int(t[1]) for t in tiles] == [s[1] for s in segs]
+    for (start, ln, k0s, k0l, k1s, k1l, vis_end, work), (s0, l0, _, g, seg) in zip(tiles.tolist(), segs):
+        gs = [x for x in segs if x[3] == g and x[4] == 0][0]
+        gend = max(x[0] + x[1] for x in segs if x[3] == g)
+        if seg == 0:
+            assert (k0s, k0l, k1l, vis_end) == (gs[0], 0, 0, gend)
+        else:
+            assert (k0s, k0l, k1s, k1l, vis_end) == (gs[0], gs[1], s0, 0, s0 + l0)
+    units = plan.read_bwd_units(n)
+    assert sorted(map(tuple, units.tolist())) == [(h, t) for h in range(2) for t in range(n)]
+    for j in range(0, w.total_tokens, 97):
+        seg = [x for x in segs if x[0] <= j < x[0] + x[1]][0]
+        gend = max(x[0] + x[1] for x in segs if x[3] == seg[3])
+        assert key_end[j] == (gend if seg[4] == 0 else seg[0] + seg[1])
+
+
 def test_device_side_validation_reports_status():
     from paper_2602_24082_b200 import binding as B
     w = W.Workload("bad", [[(5, (2, 4))], [(3, (1, 2))]], 2, 1, 64, seed=0)
