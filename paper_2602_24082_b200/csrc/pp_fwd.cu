@@ -303,8 +303,13 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         const int col_lim = kt.diag ? min(kt.len, row + 1) : kt.len;
         float mx = -INFINITY;
         if (full) {
+          float m1 = -INFINITY;  // two chains of three-input maxima
 #pragma unroll
-          for (int i = 0; i < 128; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
+          for (int i = 0; i < 128; i += 4) {
+            mx = max3(mx, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+            m1 = max3(m1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+          }
+          mx = fmaxf(mx, m1);
         } else {
 #pragma unroll
           for (int i = 0; i < 128; ++i)
@@ -336,13 +341,20 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         float rs = 0.f;
         const float neg_m = -m_used;
         if (full) {
+          // packed pairs: one FMA and one ADD instruction per two elements
+          const uint64_t sc2 = pack2(prm.scale_log2, prm.scale_log2), nm2 = pack2(neg_m, neg_m);
+          uint64_t sum2 = pack2(0.f, 0.f);
 #pragma unroll
           for (int i = 0; i < 64; ++i) {
-            const float p0 = ex2(fmaf(__uint_as_float(v[2 * i]), prm.scale_log2, neg_m));
-            const float p1 = ex2(fmaf(__uint_as_float(v[2 * i + 1]), prm.scale_log2, neg_m));
-            rs += p0 + p1;
+            float x0, x1;
+            unpack2(fma2(pack2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), sc2, nm2), x0, x1);
+            const float p0 = ex2(x0), p1 = ex2(x1);
+            sum2 = add2(sum2, pack2(p0, p1));
             v[i] = pack_bf16(p0, p1);
           }
+          float s0, s1;
+          unpack2(sum2, s0, s1);
+          rs = s0 + s1;
         } else {
 #pragma unroll
           for (int i = 0; i < 64; ++i) {
