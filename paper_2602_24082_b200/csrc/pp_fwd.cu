@@ -4,13 +4,15 @@
 //   warp 0      TMA producer: Q tiles of the unit's two query heads, then the K / V tiles of
 //               every visible key tile through two-stage rings
 //   warp 1      MMA issuer (one thread): S = Q K^T and O += P V with tcgen05.mma, fp32 in TMEM
-//   warps 2-5   softmax warpgroup of slot 0: thread = query row = TMEM lane
-//   warps 6-9   softmax warpgroup of slot 1
+//   warps 2-9   softmax warps of slot 0: two threads per query row (= TMEM lane), 64 key
+//               columns each
+//   warps 10-17 softmax warps of slot 1
 // A work unit is (query tile, KV head, pair of query heads of that KV head): both slots see
 // the same keys and the same mask, so every K / V tile staged in shared memory feeds two
 // S tiles.  While one slot's warpgroup does its exponentials the tensor core works on the
-// other slot (order: PV_0(j), QK_0(j+1), PV_1(j), QK_1(j+1), ...).  P (bf16) overwrites the
-// first 64 columns of its S tile in tensor memory and is the A operand of the second MMA; V is
+// other slot (order: PV_0(j), QK_0(j+1), PV_1(j), QK_1(j+1), ...).  P (bf16) overwrites columns
+// [0,32) and [64,96) of its S tile in tensor memory (each half-row thread inside the columns it
+// has read itself) and is the A operand of the second MMA; V is
 // its MN-major B operand straight from the TMA layout.  O is rescaled lazily: only when a
 // row's running maximum grew by more than 2^8 since the value used for scaling.
 // TMEM: S0 | S1 | O0 | O1, 128 columns each.
@@ -31,7 +33,7 @@ struct FwdParams {
   float scale_log2;  // softmax scale * log2(e)
 };
 
-constexpr int kFwdThreads = 320;
+constexpr int kFwdThreads = 576;
 constexpr uint32_t kFwdTmemCols = 512;
 constexpr float kRescaleThreshold = 8.f;  // log2 units
 
@@ -47,7 +49,7 @@ enum FwdBar : int {
   kODone = 16,
   kOFree = 18,
   kSchedFullF = 20,   // [2] unit ids handed from the producer to the other roles
-  kSchedEmptyF = 22,  // [2] 9 arrivals: MMA thread + 8 softmax warps
+  kSchedEmptyF = 22,  // [2] 17 arrivals: MMA thread + 16 softmax warps
   kNumFwdBars = 24
 };
 
@@ -55,7 +57,8 @@ template <int D>
 struct FwdSmem {
   static constexpr int kTileBytes = 128 * D * 2;
   static constexpr int kQ = 0, kK = 2 * kTileBytes, kV = 4 * kTileBytes, kBars = 6 * kTileBytes;
-  static constexpr int kTotal = kBars + 256 + 1024;  // + slack to align the base to 1024 B
+  static constexpr int kXch = kBars + 256;            // float [2 slots][2 buffers][128 rows][2 halves]
+  static constexpr int kTotal = kXch + 4096 + 1024;   // + slack to align the base to 1024 B
 };
 
 struct KvTile {
@@ -135,7 +138,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     for (int i = 0; i < kNumFwdBars; ++i) {
       const bool wg_count = (i >= kPFull && i < kPFull + 2) || (i >= kOFree && i < kOFree + 2);
       const bool sched_empty = (i >= kSchedEmptyF && i < kSchedEmptyF + 2);
-      mbar_init(bar(i), wg_count ? 128 : (sched_empty ? 9 : 1));
+      mbar_init(bar(i), wg_count ? 256 : (sched_empty ? 17 : 1));
     }
     *abort_flag = 0;
     fence_mbar_init();
@@ -260,7 +263,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk)
               if (kk < ksteps)
-                mma_ts(tmem + 256 + s * 128, tmem + s * 128 + kk * 8, dv + mnmajor_off(kk), idesc_o,
+                mma_ts(tmem + 256 + s * 128, tmem + s * 128 + (kk < 4 ? kk * 8 : 64 + (kk - 4) * 8), dv + mnmajor_off(kk), idesc_o,
                        (j > 0) || (kk > 0));
             mma_commit(bar(kODone + s));
             ++tc[s];
@@ -281,71 +284,85 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       }
     }
   } else {
-    // ------------------------------------------------------------ softmax warpgroups
-    const int s = (warp - 2) >> 2;
-    const int row = 32 * (warp & 3) + lane;
-    const uint32_t lane_base = tmem + (uint32_t(32 * (warp & 3)) << 16);
-    const uint32_t tS = lane_base + s * 128, tO = lane_base + 256 + s * 128;
+    // ------------------------------------------------------------ softmax warps
+    // Eight warps per slot: two threads share a query row (= TMEM lane), each owning 64 of
+    // the tile's 128 key columns and D/2 of the output columns.  Halving the work per thread
+    // keeps one slot's softmax shorter than the other slot's MMA phase, so the two slots'
+    // exponentials do not pile up on the same MUFU at the same time.  The two halves of a row
+    // exchange their partial maxima (every tile) and sums (once per unit) through shared
+    // memory, guarded by a 64-thread named barrier per (slot, lane quarter).
+    const int lw = warp - 2;                  // 0..15
+    const int s = lw >> 3;                    // slot
+    const int half = (lw >> 2) & 1;           // column half of the row
+    const int qd = warp & 3;                  // lane quarter this warp may touch
+    const int row = 32 * qd + lane;
+    const int bar_id = 1 + s * 4 + qd;        // named barrier shared with the partner warp
+    const uint32_t lane_base = tmem + (uint32_t(32 * qd) << 16);
+    const uint32_t tS = lane_base + s * 128 + half * 64;   // my S columns; P goes to their start
+    const uint32_t tO = lane_base + 256 + s * 128 + half * (D / 2);
+    float* xch = reinterpret_cast<float*>(gbase + L::kXch) + s * 512;  // [2 buffers][128 rows][2]
     uint32_t tcS = 0;
     Unit un;
     for (uint32_t un_i = 0; get_unit(prm, take_unit(un_i, true), ntiles_total, un); ++un_i) {
       if (s >= un.nslots) continue;
-      float m_used = -INFINITY, l_run = 0.f;
+      float m_used = -INFINITY, l_part = 0.f;
       for (int j = 0; j < un.ntiles; ++j) {
         const KvTile kt = kv_tile_of(un.tile, j, un.n0, un.n1);
         wait_bar(bar(kSFull + s), tcS & 1, abort_flag, prm.header, 40 + s);
         tc_fence_after();
-        uint32_t v[128];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[c * 32]));
+        uint32_t v[64];
+        tmem_ld32(tS, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+        tmem_ld32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
         tmem_wait_ld();
         const bool full = !kt.diag && kt.len == kTile;
-        const int col_lim = kt.diag ? min(kt.len, row + 1) : kt.len;
-        float mx = -INFINITY;
+        // visible columns of this half: [0, col_lim) in the half's own numbering
+        const int col_lim = (kt.diag ? min(kt.len, row + 1) : kt.len) - 64 * half;
+        float mx = -INFINITY, m1 = -INFINITY;
         if (full) {
-          float m1 = -INFINITY;  // two chains of three-input maxima
 #pragma unroll
-          for (int i = 0; i < 128; i += 4) {
+          for (int i = 0; i < 64; i += 4) {
             mx = max3(mx, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
             m1 = max3(m1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
           }
           mx = fmaxf(mx, m1);
         } else {
 #pragma unroll
-          for (int i = 0; i < 128; ++i)
-            mx = fmaxf(mx, i < col_lim ? __uint_as_float(v[i]) : -INFINITY);
+          for (int i = 0; i < 64; ++i) mx = fmaxf(mx, i < col_lim ? __uint_as_float(v[i]) : -INFINITY);
         }
-        mx *= prm.scale_log2;
+        // exchange the half-row maxima with the partner thread
+        float* xb = xch + (tcS & 1) * 256 + row * 2;
+        xb[half] = mx;
+        named_barrier_sync(bar_id, 64);
+        mx = fmaxf(mx, xb[half ^ 1]) * prm.scale_log2;
         if (j == 0) {
           m_used = mx;
         } else {
           const float m_new = fmaxf(m_used, mx);
           const bool need = (m_new - m_used) > kRescaleThreshold;
-          if (__any_sync(0xffffffffu, need)) {
+          if (__any_sync(0xffffffffu, need)) {  // same rows, same values in the partner warp
             const float alpha = ex2(m_used - m_new);
             wait_bar(bar(kODone + s), (tcS - 1) & 1, abort_flag, prm.header, 42 + s);
             tc_fence_after();
 #pragma unroll 1
-            for (int c = 0; c < D / 32; ++c) {
-              uint32_t w[32];
-              tmem_ld32(tO + c * 32, w);
+            for (int c = 0; c < D / 16; ++c) {  // rare path: eight columns at a time
+              uint32_t w[8];
+              tmem_ld8(tO + c * 8, w);
               tmem_wait_ld();
 #pragma unroll
-              for (int i = 0; i < 32; ++i) w[i] = __float_as_uint(__uint_as_float(w[i]) * alpha);
-              tmem_st32(tO + c * 32, w);
+              for (int i = 0; i < 8; ++i) w[i] = __float_as_uint(__uint_as_float(w[i]) * alpha);
+              tmem_st8(tO + c * 8, w);
             }
-            l_run *= alpha;
+            l_part *= alpha;
             m_used = m_new;
           }
         }
-        float rs = 0.f;
+        float rs;
         const float neg_m = -m_used;
         if (full) {
-          // packed pairs: one FMA and one ADD instruction per two elements
           const uint64_t sc2 = pack2(prm.scale_log2, prm.scale_log2), nm2 = pack2(neg_m, neg_m);
           uint64_t sum2 = pack2(0.f, 0.f);
 #pragma unroll
-          for (int i = 0; i < 64; ++i) {
+          for (int i = 0; i < 32; ++i) {
             float x0, x1;
             unpack2(fma2(pack2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), sc2, nm2), x0, x1);
             const float p0 = ex2(x0), p1 = ex2(x1);
@@ -356,8 +373,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           unpack2(sum2, s0, s1);
           rs = s0 + s1;
         } else {
+          rs = 0.f;
 #pragma unroll
-          for (int i = 0; i < 64; ++i) {
+          for (int i = 0; i < 32; ++i) {
             float p0 = ex2(fmaf(__uint_as_float(v[2 * i]), prm.scale_log2, neg_m));
             float p1 = ex2(fmaf(__uint_as_float(v[2 * i + 1]), prm.scale_log2, neg_m));
             p0 = (2 * i < col_lim) ? p0 : 0.f;
@@ -366,21 +384,24 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             v[i] = pack_bf16(p0, p1);
           }
         }
-        l_run += rs;
-        tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
-        tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
+        l_part += rs;
+        tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));  // P over my own S columns
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(bar(kPFull + s));
         ++tcS;
       }
-      // ---- epilogue: O / l -> bf16 registers, release the accumulator, then store
+      // ---- epilogue: row sum from both halves, O / l -> bf16, release the accumulator, store
+      float* xb = xch + (tcS & 1) * 256 + row * 2;
+      xb[half] = l_part;
+      named_barrier_sync(bar_id, 64);
+      const float l_run = l_part + xb[half ^ 1];
       wait_bar(bar(kODone + s), (tcS - 1) & 1, abort_flag, prm.header, 44 + s);
       tc_fence_after();
       const float inv_l = 1.f / l_run;
-      uint32_t ob[D / 2];
+      uint32_t ob[D / 4];
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
+      for (int c = 0; c < D / 64; ++c) {
         uint32_t w[32];
         tmem_ld32(tO + c * 32, w);
         tmem_wait_ld();
@@ -390,13 +411,15 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       }
       tc_fence_before();
       mbar_arrive(bar(kOFree + s));
+      // the exchange buffer of parity (tcS & 1) is written again two uses later, after another
+      // barrier: no further synchronisation needed here
       if (row < un.tile.len) {
         const int h = un.h0 + s;
         const size_t tok = size_t(un.tile.start) + row;
-        prm.lse[size_t(h) * prm.T + tok] = (m_used + log2f(l_run)) * 0.69314718055994531f;
-        uint4* dst = reinterpret_cast<uint4*>(prm.o + (tok * prm.Hq + h) * D);
+        if (half == 0) prm.lse[size_t(h) * prm.T + tok] = (m_used + log2f(l_run)) * 0.69314718055994531f;
+        uint4* dst = reinterpret_cast<uint4*>(prm.o + (tok * prm.Hq + h) * D + half * (D / 2));
 #pragma unroll
-        for (int i = 0; i < D / 8; ++i)
+        for (int i = 0; i < D / 16; ++i)
           dst[i] = make_uint4(ob[4 * i], ob[4 * i + 1], ob[4 * i + 2], ob[4 * i + 3]);
       }
     }
