@@ -199,7 +199,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 
   if (prm.header[0] != kStatusOk) return;
   const int ntiles_total = prm.header[2];
-#ifdef PP_TIMING
+#ifdef PP_DEBUG_COUNTERS
   const long long t_kernel0 = clock64();
 #endif
 
@@ -591,13 +591,13 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       prm.header[kHdrBwdDone] = 0;
     }
   }
-#ifdef PP_TIMING
+#ifdef PP_DEBUG_COUNTERS
   if (blockIdx.x == 0 && tid == 0) g_wait_cycles[127] = (unsigned long long)(clock64() - t_kernel0);
   if (tid == 0) g_cta_cycles[blockIdx.x & 255] = (unsigned long long)(clock64() - t_kernel0);
 #endif
 }
 
-#ifdef PP_TIMING
+#ifdef PP_DEBUG_COUNTERS
 }  // namespace
 }  // namespace pp
 extern "C" int pp_debug_bwd_cta_cycles(unsigned long long* out) {

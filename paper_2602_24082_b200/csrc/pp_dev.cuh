@@ -13,9 +13,12 @@ constexpr uint32_t kSpinLimit = 1u << 21;  // polls of mbarrier.try_wait before 
 // Waits for a phase of an mbarrier, but never forever: after kSpinLimit polls the CTA records
 // the site in the plan's status word, raises its abort flag (which turns every later wait of
 // this CTA into a no-op) and carries on to its normal exit path.
-#ifdef PP_TIMING
-// Developer switch (-DPP_TIMING): cycles CTA 0 spends in each wait site, summed over lane 0
-// of every warp that waits there; slot 127 holds CTA 0's total cycles.
+#if defined(PP_TIMING) || defined(PP_CYCLES)
+// Developer switches.  -DPP_TIMING: cycles CTA 0 spends in each wait site, summed over lane 0
+// of every warp that waits there (the waits lose their fast path, so totals are inflated);
+// slot 127 holds CTA 0's total cycles.  -DPP_CYCLES: only the per-CTA total cycles, with the
+// kernels otherwise unchanged.
+#define PP_DEBUG_COUNTERS 1
 static __device__ unsigned long long g_wait_cycles[128];
 static __device__ unsigned long long g_cta_cycles[256];  // per-CTA busy cycles
 #endif

@@ -17,6 +17,7 @@
 // row's running maximum grew by more than 2^8 since the value used for scaling.
 // TMEM: S0 | S1 | O0 | O1, 128 columns each.
 #include <algorithm>
+#include <type_traits>
 
 #include "pp_dev.cuh"
 
@@ -121,7 +122,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 
   if (prm.header[0] != kStatusOk) return;
   const int ntiles_total = prm.header[2];
-#ifdef PP_TIMING
+#ifdef PP_DEBUG_COUNTERS
   const long long t_kernel0 = clock64();
 #endif
 
@@ -219,66 +220,107 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
+    // tcgen05.mma issue blocks this thread for about one MMA duration, so the tensor pipe is
+    // idle whenever the thread executes anything else for longer than that: the loop below
+    // keeps the work between two groups of MMAs to a minimum (descriptors and instruction
+    // descriptors precomputed, barrier addresses and parities kept in registers, one branch
+    // for the common case of full 128-key tiles).
     if (lane == 0) {
       uint32_t kc = 0, vc = 0, tc[2] = {0, 0}, uc[2] = {0, 0};
       constexpr uint32_t idesc_o = make_idesc(128, D, 0, 1);
-      Unit un;
-      const uint64_t dq0 = kmajor_base(sQ), dk0 = kmajor_base(sK), dv0 = mnmajor_base(sV);
+      constexpr uint32_t idesc_full = make_idesc(128, 128, 0, 0);
       constexpr uint64_t kStageStep = uint64_t(L::kTileBytes >> 4);
+      const uint64_t dq[2] = {kmajor_base(sQ), kmajor_base(sQ) + kStageStep};
+      const uint64_t dk[2] = {kmajor_base(sK), kmajor_base(sK) + kStageStep};
+      const uint64_t dv[2] = {mnmajor_base(sV), mnmajor_base(sV) + kStageStep};
+      const uint32_t tSs[2] = {tmem, tmem + 128}, tOs[2] = {tmem + 256, tmem + 384};
+      // length of key tile j of a unit: only the last tile of each visible range and the
+      // diagonal tile can be shorter than 128
+      auto len_of = [](const Unit& u, int j) -> int {
+        if (j + 1 == u.n0) return u.tile.kv0_len - (u.n0 - 1) * kTile;
+        if (j + 1 == u.n0 + u.n1) return u.tile.kv1_len - (u.n1 - 1) * kTile;
+        if (j == u.n0 + u.n1) return u.tile.len;
+        return kTile;
+      };
       auto issue_qk = [&](int s, uint32_t kstage, int k_len) {
-        const uint32_t idesc_s = k_len == kTile ? make_idesc(128, 128, 0, 0)
-                                                : make_idesc(128, ((k_len + 15) >> 4) << 4, 0, 0);
-        const uint64_t dq = dq0 + s * kStageStep, dk = dk0 + kstage * kStageStep;
+        const uint64_t a = dq[s], b = kstage ? dk[1] : dk[0];
+        if (k_len == kTile) {
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk)
-          mma_ss(tmem + s * 128, dq + kmajor_off(kk), dk + kmajor_off(kk), idesc_s, kk > 0);
+          for (int kk = 0; kk < D / 16; ++kk)
+            mma_ss(tSs[s], a + kmajor_off(kk), b + kmajor_off(kk), idesc_full, kk > 0);
+        } else {
+          const uint32_t idesc_s = make_idesc(128, 0, 0, 0) | (uint32_t(((k_len + 15) >> 4) << 1) << 17);
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk)
+            mma_ss(tSs[s], a + kmajor_off(kk), b + kmajor_off(kk), idesc_s, kk > 0);
+        }
         mma_commit(bar(kSFull + s));
       };
+      auto issue_pv = [&](int s, uint32_t vstage, int k_len, bool first) {
+        const uint64_t b = vstage ? dv[1] : dv[0];
+        const uint32_t tS = tSs[s], tO = tOs[s];
+        if (k_len == kTile && !first) {
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)
+            mma_ts(tO, tS + (kk < 4 ? kk * 8 : 64 + (kk - 4) * 8), b + mnmajor_off(kk), idesc_o, 1);
+        } else {
+          const int ksteps = (k_len + 15) >> 4;
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)
+            if (kk < ksteps)
+              mma_ts(tO, tS + (kk < 4 ? kk * 8 : 64 + (kk - 4) * 8), b + mnmajor_off(kk), idesc_o,
+                     !first || (kk > 0));
+        }
+        mma_commit(bar(kODone + s));
+      };
+      Unit un;
       for (uint32_t un_i = 0; get_unit(prm, take_unit(un_i, false), ntiles_total, un); ++un_i) {
         for (int s = 0; s < un.nslots; ++s)
           wait_bar(bar(kQFull + s), uc[s] & 1, abort_flag, prm.header, 30 + s);
-        KvTile kt = kv_tile_of(un.tile, 0, un.n0, un.n1);
+        int cur_len = len_of(un, 0);
         wait_bar(bar(kKFull + (kc & 1)), (kc >> 1) & 1, abort_flag, prm.header, 32);
         tc_fence_after();
         for (int s = 0; s < un.nslots; ++s) {
-          issue_qk(s, kc & 1, kt.len);
+          issue_qk(s, kc & 1, cur_len);
           if (un.ntiles == 1) mma_commit(bar(kQEmpty + s));
         }
         mma_commit(bar(kKEmpty + (kc & 1)));
         ++kc;
+        const bool two = un.nslots == 2;
         for (int j = 0; j < un.ntiles; ++j) {
           const bool has_next = j + 1 < un.ntiles;
-          const int cur_len = kt.len;
-          KvTile nx = kt;
-          if (has_next) nx = kv_tile_of(un.tile, j + 1, un.n0, un.n1);
-          wait_bar(bar(kVFull + (vc & 1)), (vc >> 1) & 1, abort_flag, prm.header, 33);
-          if (has_next)
-            wait_bar(bar(kKFull + (kc & 1)), (kc >> 1) & 1, abort_flag, prm.header, 34);
-          const uint64_t dv = dv0 + (vc & 1) * kStageStep;
-          for (int s = 0; s < un.nslots; ++s) {
-            wait_bar(bar(kPFull + s), tc[s] & 1, abort_flag, prm.header, 35 + s);
-            if (j == 0) wait_bar(bar(kOFree + s), (uc[s] & 1) ^ 1, abort_flag, prm.header, 37 + s);
+          const int nx_len = has_next ? len_of(un, j + 1) : 0;
+          const uint32_t vst = vc & 1, kst = kc & 1;
+          wait_bar(bar(kVFull + vst), (vc >> 1) & 1, abort_flag, prm.header, 33);
+          if (has_next) wait_bar(bar(kKFull + kst), (kc >> 1) & 1, abort_flag, prm.header, 34);
+          // slot 0
+          wait_bar(bar(kPFull + 0), tc[0] & 1, abort_flag, prm.header, 35);
+          if (j == 0) wait_bar(bar(kOFree + 0), (uc[0] & 1) ^ 1, abort_flag, prm.header, 37);
+          tc_fence_after();
+          issue_pv(0, vst, cur_len, j == 0);
+          ++tc[0];
+          if (has_next) {
+            issue_qk(0, kst, nx_len);
+            if (j + 2 == un.ntiles) mma_commit(bar(kQEmpty + 0));
+          }
+          if (two) {
+            wait_bar(bar(kPFull + 1), tc[1] & 1, abort_flag, prm.header, 36);
+            if (j == 0) wait_bar(bar(kOFree + 1), (uc[1] & 1) ^ 1, abort_flag, prm.header, 38);
             tc_fence_after();
-            const int ksteps = (cur_len + 15) >> 4;
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-              if (kk < ksteps)
-                mma_ts(tmem + 256 + s * 128, tmem + s * 128 + (kk < 4 ? kk * 8 : 64 + (kk - 4) * 8), dv + mnmajor_off(kk), idesc_o,
-                       (j > 0) || (kk > 0));
-            mma_commit(bar(kODone + s));
-            ++tc[s];
+            issue_pv(1, vst, cur_len, j == 0);
+            ++tc[1];
             if (has_next) {
-              issue_qk(s, kc & 1, nx.len);
-              if (j + 2 == un.ntiles) mma_commit(bar(kQEmpty + s));
+              issue_qk(1, kst, nx_len);
+              if (j + 2 == un.ntiles) mma_commit(bar(kQEmpty + 1));
             }
           }
-          mma_commit(bar(kVEmpty + (vc & 1)));
+          mma_commit(bar(kVEmpty + vst));
           ++vc;
           if (has_next) {
-            mma_commit(bar(kKEmpty + (kc & 1)));
+            mma_commit(bar(kKEmpty + kst));
             ++kc;
           }
-          kt = nx;
+          cur_len = nx_len;
         }
         for (int s = 0; s < un.nslots; ++s) ++uc[s];
       }
@@ -413,14 +455,45 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       mbar_arrive(bar(kOFree + s));
       // the exchange buffer of parity (tcS & 1) is written again two uses later, after another
       // barrier: no further synchronisation needed here
-      if (row < un.tile.len) {
-        const int h = un.h0 + s;
-        const size_t tok = size_t(un.tile.start) + row;
-        if (half == 0) prm.lse[size_t(h) * prm.T + tok] = (m_used + log2f(l_run)) * 0.69314718055994531f;
-        uint4* dst = reinterpret_cast<uint4*>(prm.o + (tok * prm.Hq + h) * D + half * (D / 2));
+      const int h = un.h0 + s;
+      if (half == 0 && row < un.tile.len)
+        prm.lse[size_t(h) * prm.T + un.tile.start + row] = (m_used + log2f(l_run)) * 0.69314718055994531f;
+      // A thread holds kCh 16-byte chunks of one row; transposing them inside groups of kCh
+      // lanes gives every lane the same chunk of kCh consecutive rows, so that one store
+      // instruction of the warp writes whole contiguous half-rows instead of 32 scattered
+      // 16-byte pieces.
+      constexpr int kCh = D / 16;
+      auto exchange = [&](auto dist) {
+        constexpr int d = decltype(dist)::value;
+        if constexpr (d < kCh) {
+          const bool hi = (lane & d) != 0;
 #pragma unroll
-        for (int i = 0; i < D / 16; ++i)
-          dst[i] = make_uint4(ob[4 * i], ob[4 * i + 1], ob[4 * i + 2], ob[4 * i + 3]);
+          for (int i = 0; i < kCh; ++i) {
+            if ((i & d) == 0) {
+#pragma unroll
+              for (int c = 0; c < 4; ++c) {
+                const uint32_t send = hi ? ob[4 * i + c] : ob[4 * (i | d) + c];
+                const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, d);
+                if (hi) ob[4 * i + c] = recv; else ob[4 * (i | d) + c] = recv;
+              }
+            }
+          }
+        }
+      };
+      exchange(std::integral_constant<int, 4>{});
+      exchange(std::integral_constant<int, 2>{});
+      exchange(std::integral_constant<int, 1>{});
+      {
+        const int grp = lane / kCh, chunk = lane % kCh;
+#pragma unroll
+        for (int i = 0; i < kCh; ++i) {
+          const int r = 32 * qd + grp * kCh + i;
+          if (r < un.tile.len) {
+            uint4* dst = reinterpret_cast<uint4*>(
+                prm.o + ((size_t(un.tile.start) + r) * prm.Hq + h) * D + half * (D / 2) + chunk * 8);
+            *dst = make_uint4(ob[4 * i], ob[4 * i + 1], ob[4 * i + 2], ob[4 * i + 3]);
+          }
+        }
       }
     }
   }
@@ -435,13 +508,13 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       prm.header[kHdrFwdDone] = 0;
     }
   }
-#ifdef PP_TIMING
+#ifdef PP_DEBUG_COUNTERS
   if (blockIdx.x == 0 && tid == 0) g_wait_cycles[127] = (unsigned long long)(clock64() - t_kernel0);
   if (tid == 0) g_cta_cycles[blockIdx.x & 255] = (unsigned long long)(clock64() - t_kernel0);
 #endif
 }
 
-#ifdef PP_TIMING
+#ifdef PP_DEBUG_COUNTERS
 }  // namespace
 }  // namespace pp
 extern "C" int pp_debug_fwd_cta_cycles(unsigned long long* out) {
