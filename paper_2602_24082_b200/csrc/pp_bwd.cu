@@ -15,6 +15,8 @@
 #include <algorithm>
 #include <mutex>
 
+#include <type_traits>
+
 #include "pp_dev.cuh"
 
 namespace pp {
@@ -510,12 +512,49 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       }
       tc_fence_before();
       mbar_arrive(bar(kDkvFree));
-      if (row_ok) {
-        __nv_bfloat16* out = wg ? prm.dk : prm.dv;
-        uint4* dst = reinterpret_cast<uint4*>(out + ((size_t(un.tile.start) + row) * prm.Hkv + un.kvh) * D);
+      // A thread holds one row as 16-byte chunks; transposing each group of eight chunks
+      // (128 bytes) inside groups of eight lanes gives every lane the same chunk of eight
+      // consecutive rows, so that one store instruction of the warp writes four whole
+      // 128-byte lines instead of 32 scattered 16-byte pieces (which kept the SM's memory
+      // pipe busy for thousands of cycles at every unit boundary).
 #pragma unroll
-        for (int i = 0; i < D / 8; ++i)
-          dst[i] = make_uint4(ob[4 * i], ob[4 * i + 1], ob[4 * i + 2], ob[4 * i + 3]);
+      for (int hb = 0; hb < D / 64; ++hb) {
+        uint32_t* x = ob + 32 * hb;
+        auto exchange = [&](auto dist) {
+          constexpr int d = decltype(dist)::value;
+          const bool hi = (lane & d) != 0;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            if ((i & d) == 0) {
+#pragma unroll
+              for (int c = 0; c < 4; ++c) {
+                const uint32_t send = hi ? x[4 * i + c] : x[4 * (i | d) + c];
+                const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, d);
+                if (hi) x[4 * i + c] = recv; else x[4 * (i | d) + c] = recv;
+              }
+            }
+          }
+        };
+        exchange(std::integral_constant<int, 4>{});
+        exchange(std::integral_constant<int, 2>{});
+        exchange(std::integral_constant<int, 1>{});
+      }
+      {
+        __nv_bfloat16* out = wg ? prm.dk : prm.dv;
+        const int grp = lane >> 3, chunk = lane & 7;
+#pragma unroll
+        for (int hb = 0; hb < D / 64; ++hb) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int r = 32 * (warp & 3) + grp * 8 + i;
+            if (r < un.tile.len) {
+              uint4* dst = reinterpret_cast<uint4*>(
+                  out + ((size_t(un.tile.start) + r) * prm.Hkv + un.kvh) * D + hb * 64 + chunk * 8);
+              *dst = make_uint4(ob[32 * hb + 4 * i], ob[32 * hb + 4 * i + 1], ob[32 * hb + 4 * i + 2],
+                                ob[32 * hb + 4 * i + 3]);
+            }
+          }
+        }
       }
     }
   } else {

@@ -1,8 +1,10 @@
 // Forward kernel: O = softmax(mask(scale Q K^T)) V and LSE over the plan's visible tiles.
 //
 // Persistent, warp-specialised CTA (one per SM):
-//   warp 0      TMA producer: Q tiles of the unit's two query heads, then the K / V tiles of
-//               every visible key tile through two-stage rings
+//   warp 0      TMA producer: draws and decodes the work units (the only reader of the plan's
+//               tile list; the other roles get a decoded record through shared memory), loads
+//               the Q tiles of the unit's two query heads, then the K / V tiles of every
+//               visible key tile through two-stage rings
 //   warp 1      MMA issuer (one thread): S = Q K^T and O += P V with tcgen05.mma, fp32 in TMEM
 //   warps 2-9   softmax warps of slot 0: two threads per query row (= TMEM lane), 64 key
 //               columns each
@@ -58,7 +60,8 @@ template <int D>
 struct FwdSmem {
   static constexpr int kTileBytes = 128 * D * 2;
   static constexpr int kQ = 0, kK = 2 * kTileBytes, kV = 4 * kTileBytes, kBars = 6 * kTileBytes;
-  static constexpr int kXch = kBars + 256;            // float [2 slots][2 buffers][128 rows][2 halves]
+  static constexpr int kSched = kBars + 256;          // two decoded unit records of 8 ints
+  static constexpr int kXch = kSched + 64;            // float [2 slots][2 buffers][128 rows][2 halves]
   static constexpr int kTotal = kXch + 4096 + 1024;   // + slack to align the base to 1024 B
 };
 
@@ -155,24 +158,43 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot_p;
-  volatile int* sched = reinterpret_cast<volatile int*>(gbase + L::kBars + 8 * kNumFwdBars + 16);
-  auto fetch_unit = [&](uint32_t n) -> int {  // producer thread
+  // Ring of two decoded unit records (producer -> MMA thread and softmax warps): the producer
+  // alone reads the plan's tile list; the other roles get what they need from shared memory.
+  volatile int* sched = reinterpret_cast<volatile int*>(gbase + L::kSched);
+  auto fetch_unit = [&](uint32_t n, Unit& un) -> bool {  // producer thread
     wait_bar(bar(kSchedEmptyF + (n & 1)), ((n >> 1) & 1) ^ 1, abort_flag, prm.header, 90);
     const int u = atomicAdd(&prm.header[kHdrFwdNext], 1);
-    sched[n & 1] = u;
+    const bool ok = get_unit(prm, u, ntiles_total, un);
+    volatile int* e = sched + (n & 1) * 8;
+    e[0] = un.tile.start;
+    e[1] = un.tile.len;
+    e[2] = un.h0;
+    e[3] = ok ? un.nslots : 0;  // 0 slots marks the end of the work list
+    e[4] = un.n0;
+    e[5] = un.n1;
+    e[6] = un.tile.kv0_len - (un.n0 - 1) * kTile;
+    e[7] = un.tile.kv1_len - (un.n1 - 1) * kTile;
     mbar_arrive(bar(kSchedFullF + (n & 1)));
-    return u;
+    return ok;
   };
-  auto take_unit = [&](uint32_t n, bool whole_warp) -> int {
-    const bool ok = wait_bar(bar(kSchedFullF + (n & 1)), (n >> 1) & 1, abort_flag, prm.header, 91);
-    const int u = ok ? sched[n & 1] : 0x7fffffff;
-    if (whole_warp) {
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(kSchedEmptyF + (n & 1)));
-    } else {
-      mbar_arrive(bar(kSchedEmptyF + (n & 1)));
-    }
-    return u;
+  // Consumers: read the record into plain scalars (kept in registers) and release the entry.
+#define PP_TAKE_UNIT(n, whole_warp)                                                              \
+  const bool u_ok = wait_bar(bar(kSchedFullF + ((n) & 1)), ((n) >> 1) & 1, abort_flag, prm.header, 91); \
+  const volatile int* u_e = sched + ((n) & 1) * 8;                                               \
+  const int u_start = u_e[0], u_len = u_e[1], u_h0 = u_e[2], u_nslots = u_ok ? u_e[3] : 0;       \
+  const int u_n0 = u_e[4], u_n1 = u_e[5], u_last0 = u_e[6], u_last1 = u_e[7];                    \
+  const int u_ntiles = u_n0 + u_n1 + 1;                                                          \
+  if (whole_warp) {                                                                              \
+    __syncwarp();                                                                                \
+    if (lane == 0) mbar_arrive(bar(kSchedEmptyF + ((n) & 1)));                                   \
+  } else {                                                                                       \
+    mbar_arrive(bar(kSchedEmptyF + ((n) & 1)));                                                  \
+  }                                                                                              \
+  (void)u_start, (void)u_len, (void)u_h0;                                                        \
+  /* keys of visible key tile j: only the last tile of a full range and the diagonal tile */    \
+  /* can be shorter than 128 */                                                                  \
+  auto u_klen = [=](int j) -> int {                                                              \
+    return (j + 1 == u_n0) ? u_last0 : (j + 1 == u_n0 + u_n1) ? u_last1 : (j + 1 == u_ntiles) ? u_len : kTile; \
   };
 
   if (warp == 0) {
@@ -180,7 +202,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     if (lane == 0) {
       uint32_t kc = 0, vc = 0, qc[2] = {0, 0};
       Unit un;
-      for (uint32_t un_i = 0; get_unit(prm, fetch_unit(un_i), ntiles_total, un); ++un_i) {
+      for (uint32_t un_i = 0; fetch_unit(un_i, un); ++un_i) {
         for (int s = 0; s < un.nslots; ++s) {
           wait_bar(bar(kQEmpty + s), (qc[s] & 1) ^ 1, abort_flag, prm.header, 20 + s);
           mbar_expect_tx(bar(kQFull + s), L::kTileBytes);
@@ -226,39 +248,31 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     // descriptors precomputed, barrier addresses and parities kept in registers, one branch
     // for the common case of full 128-key tiles).
     if (lane == 0) {
-      uint32_t kc = 0, vc = 0, tc[2] = {0, 0}, uc[2] = {0, 0};
+      uint32_t kc = 0, vc = 0, tc0 = 0, tc1 = 0, uc0 = 0, uc1 = 0;
       constexpr uint32_t idesc_o = make_idesc(128, D, 0, 1);
       constexpr uint32_t idesc_full = make_idesc(128, 128, 0, 0);
       constexpr uint64_t kStageStep = uint64_t(L::kTileBytes >> 4);
-      const uint64_t dq[2] = {kmajor_base(sQ), kmajor_base(sQ) + kStageStep};
-      const uint64_t dk[2] = {kmajor_base(sK), kmajor_base(sK) + kStageStep};
-      const uint64_t dv[2] = {mnmajor_base(sV), mnmajor_base(sV) + kStageStep};
-      const uint32_t tSs[2] = {tmem, tmem + 128}, tOs[2] = {tmem + 256, tmem + 384};
+      const uint64_t dq0 = kmajor_base(sQ), dk0 = kmajor_base(sK), dv0 = mnmajor_base(sV);
       // length of key tile j of a unit: only the last tile of each visible range and the
       // diagonal tile can be shorter than 128
-      auto len_of = [](const Unit& u, int j) -> int {
-        if (j + 1 == u.n0) return u.tile.kv0_len - (u.n0 - 1) * kTile;
-        if (j + 1 == u.n0 + u.n1) return u.tile.kv1_len - (u.n1 - 1) * kTile;
-        if (j == u.n0 + u.n1) return u.tile.len;
-        return kTile;
-      };
       auto issue_qk = [&](int s, uint32_t kstage, int k_len) {
-        const uint64_t a = dq[s], b = kstage ? dk[1] : dk[0];
+        const uint64_t a = dq0 + s * kStageStep, b = dk0 + kstage * kStageStep;
+        const uint32_t tS = tmem + s * 128;
         if (k_len == kTile) {
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk)
-            mma_ss(tSs[s], a + kmajor_off(kk), b + kmajor_off(kk), idesc_full, kk > 0);
+            mma_ss(tS, a + kmajor_off(kk), b + kmajor_off(kk), idesc_full, kk > 0);
         } else {
           const uint32_t idesc_s = make_idesc(128, 0, 0, 0) | (uint32_t(((k_len + 15) >> 4) << 1) << 17);
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk)
-            mma_ss(tSs[s], a + kmajor_off(kk), b + kmajor_off(kk), idesc_s, kk > 0);
+            mma_ss(tS, a + kmajor_off(kk), b + kmajor_off(kk), idesc_s, kk > 0);
         }
         mma_commit(bar(kSFull + s));
       };
       auto issue_pv = [&](int s, uint32_t vstage, int k_len, bool first) {
-        const uint64_t b = vstage ? dv[1] : dv[0];
-        const uint32_t tS = tSs[s], tO = tOs[s];
+        const uint64_t b = dv0 + vstage * kStageStep;
+        const uint32_t tS = tmem + s * 128, tO = tmem + 256 + s * 128;
         if (k_len == kTile && !first) {
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk)
@@ -273,45 +287,48 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         }
         mma_commit(bar(kODone + s));
       };
-      Unit un;
-      for (uint32_t un_i = 0; get_unit(prm, take_unit(un_i, false), ntiles_total, un); ++un_i) {
-        for (int s = 0; s < un.nslots; ++s)
-          wait_bar(bar(kQFull + s), uc[s] & 1, abort_flag, prm.header, 30 + s);
-        int cur_len = len_of(un, 0);
+      for (uint32_t un_i = 0;; ++un_i) {
+        PP_TAKE_UNIT(un_i, false)
+        if (u_nslots == 0) break;
+        const bool two = u_nslots == 2;
+        wait_bar(bar(kQFull + 0), uc0 & 1, abort_flag, prm.header, 30);
+        if (two) wait_bar(bar(kQFull + 1), uc1 & 1, abort_flag, prm.header, 31);
+        int cur_len = u_klen(0);
         wait_bar(bar(kKFull + (kc & 1)), (kc >> 1) & 1, abort_flag, prm.header, 32);
         tc_fence_after();
-        for (int s = 0; s < un.nslots; ++s) {
-          issue_qk(s, kc & 1, cur_len);
-          if (un.ntiles == 1) mma_commit(bar(kQEmpty + s));
+        issue_qk(0, kc & 1, cur_len);
+        if (u_ntiles == 1) mma_commit(bar(kQEmpty + 0));
+        if (two) {
+          issue_qk(1, kc & 1, cur_len);
+          if (u_ntiles == 1) mma_commit(bar(kQEmpty + 1));
         }
         mma_commit(bar(kKEmpty + (kc & 1)));
         ++kc;
-        const bool two = un.nslots == 2;
-        for (int j = 0; j < un.ntiles; ++j) {
-          const bool has_next = j + 1 < un.ntiles;
-          const int nx_len = has_next ? len_of(un, j + 1) : 0;
+        for (int j = 0; j < u_ntiles; ++j) {
+          const bool has_next = j + 1 < u_ntiles;
+          const int nx_len = has_next ? u_klen(j + 1) : 0;
           const uint32_t vst = vc & 1, kst = kc & 1;
           wait_bar(bar(kVFull + vst), (vc >> 1) & 1, abort_flag, prm.header, 33);
           if (has_next) wait_bar(bar(kKFull + kst), (kc >> 1) & 1, abort_flag, prm.header, 34);
           // slot 0
-          wait_bar(bar(kPFull + 0), tc[0] & 1, abort_flag, prm.header, 35);
-          if (j == 0) wait_bar(bar(kOFree + 0), (uc[0] & 1) ^ 1, abort_flag, prm.header, 37);
+          wait_bar(bar(kPFull + 0), tc0 & 1, abort_flag, prm.header, 35);
+          if (j == 0) wait_bar(bar(kOFree + 0), (uc0 & 1) ^ 1, abort_flag, prm.header, 37);
           tc_fence_after();
           issue_pv(0, vst, cur_len, j == 0);
-          ++tc[0];
+          ++tc0;
           if (has_next) {
             issue_qk(0, kst, nx_len);
-            if (j + 2 == un.ntiles) mma_commit(bar(kQEmpty + 0));
+            if (j + 2 == u_ntiles) mma_commit(bar(kQEmpty + 0));
           }
           if (two) {
-            wait_bar(bar(kPFull + 1), tc[1] & 1, abort_flag, prm.header, 36);
-            if (j == 0) wait_bar(bar(kOFree + 1), (uc[1] & 1) ^ 1, abort_flag, prm.header, 38);
+            wait_bar(bar(kPFull + 1), tc1 & 1, abort_flag, prm.header, 36);
+            if (j == 0) wait_bar(bar(kOFree + 1), (uc1 & 1) ^ 1, abort_flag, prm.header, 38);
             tc_fence_after();
             issue_pv(1, vst, cur_len, j == 0);
-            ++tc[1];
+            ++tc1;
             if (has_next) {
               issue_qk(1, kst, nx_len);
-              if (j + 2 == un.ntiles) mma_commit(bar(kQEmpty + 1));
+              if (j + 2 == u_ntiles) mma_commit(bar(kQEmpty + 1));
             }
           }
           mma_commit(bar(kVEmpty + vst));
@@ -322,7 +339,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           }
           cur_len = nx_len;
         }
-        for (int s = 0; s < un.nslots; ++s) ++uc[s];
+        ++uc0;
+        if (two) ++uc1;
       }
     }
   } else {
@@ -344,90 +362,116 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const uint32_t tO = lane_base + 256 + s * 128 + half * (D / 2);
     float* xch = reinterpret_cast<float*>(gbase + L::kXch) + s * 512;  // [2 buffers][128 rows][2]
     uint32_t tcS = 0;
-    Unit un;
-    for (uint32_t un_i = 0; get_unit(prm, take_unit(un_i, true), ntiles_total, un); ++un_i) {
-      if (s >= un.nslots) continue;
+    for (uint32_t un_i = 0;; ++un_i) {
+      PP_TAKE_UNIT(un_i, true)
+      if (u_nslots == 0) break;
+      if (s >= u_nslots) continue;
       float m_used = -INFINITY, l_part = 0.f;
-      for (int j = 0; j < un.ntiles; ++j) {
-        const KvTile kt = kv_tile_of(un.tile, j, un.n0, un.n1);
+      for (int j = 0; j < u_ntiles; ++j) {
+        KvTile kt;
+        kt.len = u_klen(j);
+        kt.diag = j + 1 == u_ntiles;
         wait_bar(bar(kSFull + s), tcS & 1, abort_flag, prm.header, 40 + s);
         tc_fence_after();
-        uint32_t v[64];
-        tmem_ld32(tS, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
-        tmem_ld32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
-        tmem_wait_ld();
         const bool full = !kt.diag && kt.len == kTile;
         // visible columns of this half: [0, col_lim) in the half's own numbering
         const int col_lim = (kt.diag ? min(kt.len, row + 1) : kt.len) - 64 * half;
-        float mx = -INFINITY, m1 = -INFINITY;
-        if (full) {
-#pragma unroll
-          for (int i = 0; i < 64; i += 4) {
-            mx = max3(mx, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
-            m1 = max3(m1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
-          }
-          mx = fmaxf(mx, m1);
-        } else {
-#pragma unroll
-          for (int i = 0; i < 64; ++i) mx = fmaxf(mx, i < col_lim ? __uint_as_float(v[i]) : -INFINITY);
-        }
-        // exchange the half-row maxima with the partner thread
         float* xb = xch + (tcS & 1) * 256 + row * 2;
-        xb[half] = mx;
-        named_barrier_sync(bar_id, 64);
-        mx = fmaxf(mx, xb[half ^ 1]) * prm.scale_log2;
-        if (j == 0) {
-          m_used = mx;
-        } else {
-          const float m_new = fmaxf(m_used, mx);
-          const bool need = (m_new - m_used) > kRescaleThreshold;
-          if (__any_sync(0xffffffffu, need)) {  // same rows, same values in the partner warp
-            const float alpha = ex2(m_used - m_new);
-            wait_bar(bar(kODone + s), (tcS - 1) & 1, abort_flag, prm.header, 42 + s);
-            tc_fence_after();
-#pragma unroll 1
-            for (int c = 0; c < D / 16; ++c) {  // rare path: eight columns at a time
-              uint32_t w[8];
-              tmem_ld8(tO + c * 8, w);
-              tmem_wait_ld();
+        // The 64 scores of this thread are handled as two chunks of 32 (fewer live registers).
+        // max over the visible scores of one chunk
+        auto chunk_max = [&](const uint32_t (&w)[32], int c, float m) -> float {
+          if (full) {
+            float m1 = -INFINITY;
 #pragma unroll
-              for (int i = 0; i < 8; ++i) w[i] = __float_as_uint(__uint_as_float(w[i]) * alpha);
-              tmem_st8(tO + c * 8, w);
+            for (int i = 0; i < 32; i += 4) {
+              m = max3(m, __uint_as_float(w[i]), __uint_as_float(w[i + 1]));
+              m1 = max3(m1, __uint_as_float(w[i + 2]), __uint_as_float(w[i + 3]));
             }
-            l_part *= alpha;
-            m_used = m_new;
+            return fmaxf(m, m1);
           }
+#pragma unroll
+          for (int i = 0; i < 32; ++i) m = fmaxf(m, 32 * c + i < col_lim ? __uint_as_float(w[i]) : -INFINITY);
+          return m;
+        };
+        float mx = -INFINITY;
+        bool settled = (j == 0);
+        if (settled) {
+          // first tile of the unit: the reference maximum is needed before the exponentials
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+            uint32_t w[32];
+            tmem_ld32(tS + 32 * c, w);
+            tmem_wait_ld();
+            mx = chunk_max(w, c, mx);
+          }
+          xb[half] = mx;
+          named_barrier_sync(bar_id, 64);
+          m_used = fmaxf(mx, xb[half ^ 1]) * prm.scale_log2;
         }
+        // Later tiles: the exponentials use the reference maximum of the previous tiles while
+        // the half-row maxima are exchanged; only if the new maximum exceeds the reference by
+        // more than the rescale threshold (rare) is the accumulator rescaled and the tile redone
+        // from the S values, which stay in tensor memory until P is stored.
+        uint32_t pk[32];
         float rs;
-        const float neg_m = -m_used;
-        if (full) {
+        for (;;) {
+          const float neg_m = -m_used;
           const uint64_t sc2 = pack2(prm.scale_log2, prm.scale_log2), nm2 = pack2(neg_m, neg_m);
           uint64_t sum2 = pack2(0.f, 0.f);
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            float x0, x1;
-            unpack2(fma2(pack2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), sc2, nm2), x0, x1);
-            const float p0 = ex2(x0), p1 = ex2(x1);
-            sum2 = add2(sum2, pack2(p0, p1));
-            v[i] = pack_bf16(p0, p1);
+          for (int c = 0; c < 2; ++c) {
+            uint32_t w[32];
+            tmem_ld32(tS + 32 * c, w);
+            tmem_wait_ld();
+            if (!settled) mx = chunk_max(w, c, mx);
+            if (full) {
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                float x0, x1;
+                unpack2(fma2(pack2(__uint_as_float(w[2 * i]), __uint_as_float(w[2 * i + 1])), sc2, nm2), x0, x1);
+                const float p0 = ex2(x0), p1 = ex2(x1);
+                sum2 = add2(sum2, pack2(p0, p1));
+                pk[16 * c + i] = pack_bf16(p0, p1);
+              }
+            } else {
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                float p0 = ex2(fmaf(__uint_as_float(w[2 * i]), prm.scale_log2, neg_m));
+                float p1 = ex2(fmaf(__uint_as_float(w[2 * i + 1]), prm.scale_log2, neg_m));
+                p0 = (32 * c + 2 * i < col_lim) ? p0 : 0.f;
+                p1 = (32 * c + 2 * i + 1 < col_lim) ? p1 : 0.f;
+                sum2 = add2(sum2, pack2(p0, p1));
+                pk[16 * c + i] = pack_bf16(p0, p1);
+              }
+            }
           }
           float s0, s1;
           unpack2(sum2, s0, s1);
           rs = s0 + s1;
-        } else {
-          rs = 0.f;
+          if (settled) break;
+          xb[half] = mx;
+          named_barrier_sync(bar_id, 64);
+          const float m_new = fmaxf(m_used, fmaxf(mx, xb[half ^ 1]) * prm.scale_log2);
+          const bool need = (m_new - m_used) > kRescaleThreshold;
+          if (!__any_sync(0xffffffffu, need)) break;  // same rows, same values in the partner warp
+          const float alpha = ex2(m_used - m_new);
+          wait_bar(bar(kODone + s), (tcS - 1) & 1, abort_flag, prm.header, 42 + s);
+          tc_fence_after();
+#pragma unroll 1
+          for (int c = 0; c < D / 16; ++c) {  // eight columns at a time
+            uint32_t w[8];
+            tmem_ld8(tO + c * 8, w);
+            tmem_wait_ld();
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            float p0 = ex2(fmaf(__uint_as_float(v[2 * i]), prm.scale_log2, neg_m));
-            float p1 = ex2(fmaf(__uint_as_float(v[2 * i + 1]), prm.scale_log2, neg_m));
-            p0 = (2 * i < col_lim) ? p0 : 0.f;
-            p1 = (2 * i + 1 < col_lim) ? p1 : 0.f;
-            rs += p0 + p1;
-            v[i] = pack_bf16(p0, p1);
+            for (int i = 0; i < 8; ++i) w[i] = __float_as_uint(__uint_as_float(w[i]) * alpha);
+            tmem_st8(tO + c * 8, w);
           }
+          l_part *= alpha;
+          m_used = m_new;
+          settled = true;
         }
         l_part += rs;
-        tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));  // P over my own S columns
+        tmem_st32(tS, pk);  // P over the first half of my own S columns
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(bar(kPFull + s));
@@ -455,9 +499,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       mbar_arrive(bar(kOFree + s));
       // the exchange buffer of parity (tcS & 1) is written again two uses later, after another
       // barrier: no further synchronisation needed here
-      const int h = un.h0 + s;
-      if (half == 0 && row < un.tile.len)
-        prm.lse[size_t(h) * prm.T + un.tile.start + row] = (m_used + log2f(l_run)) * 0.69314718055994531f;
+      const int h = u_h0 + s;
+      if (half == 0 && row < u_len)
+        prm.lse[size_t(h) * prm.T + u_start + row] = (m_used + log2f(l_run)) * 0.69314718055994531f;
       // A thread holds kCh 16-byte chunks of one row; transposing them inside groups of kCh
       // lanes gives every lane the same chunk of kCh consecutive rows, so that one store
       // instruction of the warp writes whole contiguous half-rows instead of 32 scattered
@@ -488,9 +532,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 #pragma unroll
         for (int i = 0; i < kCh; ++i) {
           const int r = 32 * qd + grp * kCh + i;
-          if (r < un.tile.len) {
+          if (r < u_len) {
             uint4* dst = reinterpret_cast<uint4*>(
-                prm.o + ((size_t(un.tile.start) + r) * prm.Hq + h) * D + half * (D / 2) + chunk * 8);
+                prm.o + ((size_t(u_start) + r) * prm.Hq + h) * D + half * (D / 2) + chunk * 8);
             *dst = make_uint4(ob[4 * i], ob[4 * i + 1], ob[4 * i + 2], ob[4 * i + 3]);
           }
         }
