@@ -279,21 +279,71 @@ __global__ void plan_units_kernel(PlanPtrs p) {
 }
 
 // The whole plan in one block: used when the problem is small enough that one block's
-// latency beats four dependent launches (every stage only needs block-level ordering).
+// latency beats seven dependent launches (every stage only needs block-level ordering).  The
+// per-tile keys of the rank-counting stages are kept in shared memory, so that the O(n^2)
+// loops do not go through global memory, and key_end is filled tile by tile (every key of a
+// tile ends its visibility at the tile's vis_end) instead of by a search per token.
+constexpr int kFusedMaxTiles = 2048;
+
 __global__ void __launch_bounds__(1024) plan_fused_kernel(PlanPtrs p) {
+  __shared__ uint16_t s_wf[kFusedMaxTiles];   // forward work
+  __shared__ uint16_t s_wb[kFusedMaxTiles];   // backward work
+  __shared__ int32_t s_gs[kFusedMaxTiles];    // group id (start of the group's prompt)
+  __shared__ int32_t s_gw[kFusedMaxTiles];    // backward work of the tile's whole group
+  __shared__ uint16_t s_sg[kFusedMaxTiles];   // super-group
   if (!plan_scan_body(p)) return;
   const int n = p.header[2];
-  for (int t = threadIdx.x; t < n; t += blockDim.x) plan_tile_body(p, t);
-  for (int j = threadIdx.x; j < p.T; j += blockDim.x) plan_key_end_body(p, j);
-  __syncthreads();
-  for (int t = threadIdx.x; t < n; t += blockDim.x) {
-    plan_order_body(p, t, n);
-    plan_gwork_body(p, t, n);
+  const int tid = threadIdx.x, nthr = blockDim.x;
+  for (int t = tid; t < n; t += nthr) {
+    plan_tile_body(p, t);
+    const Tile tl = p.tiles[t];  // own write
+    s_wf[t] = uint16_t(tl.work);
+    s_wb[t] = uint16_t(bwd_work(tl));
+    s_gs[t] = tl.kv0_start;
   }
   __syncthreads();
-  for (int t = threadIdx.x; t < n; t += blockDim.x) plan_sgroup_body(p, t, n);
+  // key_end: one warp per tile, coalesced
+  for (int t = tid >> 5; t < n; t += nthr >> 5) {
+    const Tile tl = p.tiles[t];
+    for (int i = tid & 31; i < tl.len; i += 32) p.key_end[tl.start + i] = tl.vis_end;
+  }
+  // longest-work-first orders by rank counting, and the work of each tile's group
+  for (int t = tid; t < n; t += nthr) {
+    const int wf = s_wf[t], wb = s_wb[t], gs = s_gs[t];
+    int rf = 0, rb = 0, gw = 0;
+    for (int u = 0; u < n; ++u) {
+      const int of = s_wf[u], ob = s_wb[u];
+      rf += (of > wf) || (of == wf && u < t);
+      rb += (ob > wb) || (ob == wb && u < t);
+      gw += (s_gs[u] == gs) ? ob : 0;
+    }
+    p.fwd_order[rf] = t;
+    p.bwd_order[rb] = t;
+    p.tile_gwork[t] = gw;
+    s_gw[t] = gw;
+  }
   __syncthreads();
-  for (int t = threadIdx.x; t < n; t += blockDim.x) plan_units_body(p, t, n);
+  for (int t = tid; t < n; t += nthr) {
+    const int gs = s_gs[t], gw = s_gw[t];
+    int rest = 0;  // tiles of this group and of the groups that come later
+    for (int u = 0; u < n; ++u) {
+      const int ogs = s_gs[u], ow = s_gw[u];
+      rest += (ogs == gs) || (ow < gw) || (ow == gw && ogs > gs);
+    }
+    const int sg = (p.Hkv * rest - 1) / kSuperGroupUnits;
+    p.tile_sgroup[t] = sg;
+    s_sg[t] = uint16_t(sg);
+  }
+  __syncthreads();
+  for (int t = tid; t < n; t += nthr) {
+    const int sg = s_sg[t], wb = s_wb[t];
+    int pos = 0;
+    for (int u = 0; u < n; ++u) {
+      const int osg = s_sg[u], ob = s_wb[u];
+      pos += (osg > sg) || (osg == sg && ((ob > wb) || (ob == wb && u < t)));
+    }
+    for (int kvh = 0; kvh < p.Hkv; ++kvh) p.bwd_units[p.Hkv * pos + kvh] = (kvh << 24) | t;
+  }
 }
 
 }  // namespace
@@ -355,7 +405,7 @@ cudaError_t launch_plan(const pp_plan* plan, cudaStream_t stream, int* launches)
   p.max_tiles = plan->max_tiles;
 
   int mt = plan->max_tiles;
-  if (mt <= 2048 && p.T <= (1 << 18)) {
+  if (mt <= kFusedMaxTiles && p.T <= (1 << 18)) {
     plan_fused_kernel<<<1, 1024, 0, stream>>>(p);
     if (launches) *launches = 1;
     return cudaGetLastError();
