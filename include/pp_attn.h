@@ -98,15 +98,25 @@ int pp_plan_status(const pp_plan* plan, pp_stream_t stream, int32_t* status, int
 /* Frees the host handle only. */
 int pp_destroy_plan(pp_plan* plan);
 
-/* Debug / test access: copies the tile table to host memory after synchronising `stream`.
- * Each tile is 8 int32: {start, len, kv0_start, kv0_len, kv1_start, kv1_len, vis_end, work}.
- * fwd_order / bwd_order receive the processing orders (tile indices).  key_end receives,
- * per token j, the first query index that can NOT see key j.  Any pointer may be NULL.
- * *num_tiles receives the tile count; arrays must hold pp_plan_max_tiles entries. */
+/* Debug / test access: copies the forward tile table to host memory after synchronising
+ * `stream`.  Each tile is 8 int32: {start, len, kv0_start, kv0_len, kv1_start, kv1_len, vis_end,
+ * work}; forward tiles are cut per segment.  fwd_order receives the forward processing order
+ * (tile indices); bwd_order the backward tiles (indices into the backward tile table, below)
+ * longest work first.  key_end receives, per token j, the first query index that can NOT see
+ * key j.  Any pointer may be NULL.  *num_tiles receives the forward tile count; arrays must
+ * hold pp_plan_max_tiles entries. */
 int pp_plan_max_tiles(const pp_plan* plan);
-/* Backward processing order: max_tiles * Hkv records (kv_head << 24) | tile, of which the
- * first num_tiles * Hkv are valid.  Units of one group are adjacent (they stream the same
- * Q / dO tiles through L2), groups with the most work first.  Synchronises `stream`. */
+/* The backward's key tiles: each GROUP (prompt and responses as one token range) cut into
+ * tiles of 128 tokens from the group's start, so a tile may straddle segments.  Each record is
+ * 8 int32: {start, len, vis_end, full_end, grp_start, grp_end, work, 0}: queries
+ * [start, vis_end) see at least one key of the tile, queries [start + len, full_end) see all
+ * of them, work = number of 128-token query tiles from `start` that reach vis_end.
+ * *num_tiles receives their count (at most pp_plan_max_tiles).  Synchronises `stream`. */
+int pp_plan_read_bwd_tiles(const pp_plan* plan, pp_stream_t stream, int32_t* num_tiles,
+                           int32_t* btiles);
+/* Backward processing order: max_tiles * Hkv records (kv_head << 24) | backward tile, of which
+ * the first num_bwd_tiles * Hkv are valid.  Units of one group are adjacent (they stream the
+ * same Q / dO tiles through L2), groups with the most work first.  Synchronises `stream`. */
 int pp_plan_read_bwd_units(const pp_plan* plan, pp_stream_t stream, int32_t* units);
 int pp_plan_read(const pp_plan* plan, pp_stream_t stream, int32_t* num_tiles, int32_t* tiles,
                  int32_t* fwd_order, int32_t* bwd_order, int32_t* key_end);

@@ -25,6 +25,7 @@ EXPORTS = ["pp_plan_workspace_bytes", "pp_build_plan", "pp_plan_status", "pp_des
            "pp_last_launch_count", "pp_error_string", "pp_step_host_arena_bytes",
            "pp_attn_step_host", "pp_profile_enable", "pp_profile_read",
            "pp_attn_bwd_noalloc", "pp_attn_bwd_noalloc_max_bytes", "pp_plan_read_bwd_units",
+           "pp_plan_read_bwd_tiles",
            "pp_position_ids", "pp_rope_qk", "pp_preference_loss"]
 
 
@@ -67,6 +68,7 @@ def lib() -> ctypes.CDLL:
         L.pp_destroy_plan.argtypes = [vp]
         L.pp_plan_max_tiles.argtypes = [vp]
         L.pp_plan_read_bwd_units.argtypes = [vp, vp, vp]
+        L.pp_plan_read_bwd_tiles.argtypes = [vp, vp, vp, vp]
         L.pp_plan_read.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         L.pp_attn_fwd.argtypes = [vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, sz, vp]
         L.pp_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, sz, vp]
@@ -130,8 +132,17 @@ class Plan:
                                   fo.ctypes.data, bo.ctypes.data, ke.ctypes.data), "pp_plan_read")
         return tiles[:n.value], fo[:n.value], bo[:n.value], ke
 
+    def read_bwd_tiles(self) -> np.ndarray:
+        """Backward key tiles [n, 8]: start, len, vis_end, full_end, grp_start, grp_end, work, 0."""
+        mt = lib().pp_plan_max_tiles(self.handle)
+        bt = np.zeros((mt, 8), dtype=np.int32)
+        n = ctypes.c_int32(0)
+        _check(lib().pp_plan_read_bwd_tiles(self.handle, _stream(), ctypes.byref(n), bt.ctypes.data),
+               "pp_plan_read_bwd_tiles")
+        return bt[:n.value]
+
     def read_bwd_units(self, num_tiles: int) -> np.ndarray:
-        """The backward processing order as (kv_head, tile) rows."""
+        """The backward processing order as (kv_head, backward tile) rows."""
         mt = lib().pp_plan_max_tiles(self.handle)
         hkv = self.problem.num_kv_heads
         raw = np.zeros(mt * hkv, dtype=np.int32)

@@ -153,6 +153,22 @@ int pp_plan_read_bwd_units(const pp_plan* plan, pp_stream_t stream, int32_t* uni
   return PP_OK;
 }
 
+int pp_plan_read_bwd_tiles(const pp_plan* plan, pp_stream_t stream, int32_t* num_tiles,
+                           int32_t* btiles) {
+  if (!plan) return PP_ERR_INVALID_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  int32_t h[16] = {};
+  bool ok = cudaMemcpyAsync(h, plan->ws + plan->lay.header, sizeof h, cudaMemcpyDeviceToHost, s) ==
+            cudaSuccess;
+  if (ok && btiles)
+    ok = cudaMemcpyAsync(btiles, plan->ws + plan->lay.btiles,
+                         size_t(plan->max_tiles) * sizeof(pp::BTile), cudaMemcpyDeviceToHost,
+                         s) == cudaSuccess;
+  if (!ok || cudaStreamSynchronize(s) != cudaSuccess) return PP_ERR_CUDA;
+  if (num_tiles) *num_tiles = h[pp::kHdrNumBTiles];
+  return h[0] == 0 ? PP_OK : PP_ERR_PLAN_STATUS;
+}
+
 int pp_plan_read(const pp_plan* plan, pp_stream_t stream, int32_t* num_tiles, int32_t* tiles,
                  int32_t* fwd_order, int32_t* bwd_order, int32_t* key_end) {
   if (!plan) return PP_ERR_INVALID_ARG;

@@ -24,8 +24,9 @@ namespace {
 
 struct BwdParams {
   int32_t* header;
-  const Tile* tiles;
+  const BTile* tiles;       // the backward's key tiles (cut per group)
   const int32_t* order;
+  const int32_t* key_end;   // [T] first query that cannot see key j
   const float* delta;  // [Hq][T]
   const float* lse2;   // [Hq][T]  LSE * log2(e)
   float* dq_acc;       // [T][Hq][D] fp32
@@ -143,7 +144,7 @@ struct BwdSmem {
 };
 
 struct BwdUnit {
-  Tile tile;
+  BTile tile;
   int kvh, nq, n_it;
 };
 
@@ -157,18 +158,20 @@ constexpr int kHdrBwdNext = 5, kHdrBwdDone = 7;
 __device__ __forceinline__ bool get_bwd_unit(const BwdParams& prm, int u, int ntiles_total,
                                              BwdUnit& un) {
   if (u < 0 || u >= ntiles_total * prm.Hkv) return false;
-  const int packed = prm.order[u];  // (kv head << 24) | tile
+  const int packed = prm.order[u];  // (kv head << 24) | backward tile
   un.kvh = packed >> 24;
   un.tile = prm.tiles[packed & 0xffffff];
-  const int full_len = un.tile.vis_end - (un.tile.start + un.tile.len);
-  un.nq = 1 + (full_len + kTile - 1) / kTile;
+  un.nq = un.tile.work;
   un.n_it = un.nq * (prm.Hq / prm.Hkv);
   return true;
 }
 
+// Query tile qt of a unit: tile qt of the group's 128-token grid counted from the key tile
+// itself.  Key j of the unit sees query i iff j <= i < key_end[j]; `full` = every key of the
+// unit sees every query of the tile and both tiles are complete (no masking code needed).
 struct QTile {
   int h, start, len;
-  bool diag;
+  bool full;
 };
 
 // (head, query tile) position inside a unit, advanced without divisions
@@ -184,9 +187,9 @@ __device__ __forceinline__ void q_advance(QIter& s, int nq) {
 __device__ __forceinline__ QTile q_tile_at(const BwdParams& prm, const BwdUnit& un, const QIter& s) {
   QTile q;
   q.h = un.kvh * (prm.Hq / prm.Hkv) + s.hh;
-  q.diag = (s.qt == 0);
-  q.start = q.diag ? un.tile.start : un.tile.start + un.tile.len + (s.qt - 1) * kTile;
-  q.len = q.diag ? un.tile.len : min(kTile, un.tile.vis_end - q.start);
+  q.start = un.tile.start + s.qt * kTile;
+  q.len = min(kTile, un.tile.grp_end - q.start);
+  q.full = s.qt > 0 && un.tile.len == kTile && q.start + kTile <= un.tile.full_end;
   return q;
 }
 
@@ -200,7 +203,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if (prm.header[0] != kStatusOk) return;
-  const int ntiles_total = prm.header[2];
+  const int ntiles_total = prm.header[kHdrNumBTiles];
 #ifdef PP_DEBUG_COUNTERS
   const long long t_kernel0 = clock64();
 #endif
@@ -415,12 +418,15 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     BwdUnit un;
     for (; get_bwd_unit(prm, take_unit(ucnt, true), ntiles_total, un); ++ucnt) {
       const bool row_ok = row < un.tile.len;
+      // my key j = tile.start + row is seen by the queries [j, key_end[j])
+      const int key_lo = un.tile.start + row;
+      const int key_hi = row_ok ? prm.key_end[key_lo] : key_lo;
       QIter qi;
       for (int it = 0; it < un.n_it; ++it, q_advance(qi, un.nq)) {
         const QTile qt = q_tile_at(prm, un, qi);
         const uint32_t g = gc + it, st = g & 1, par = g & 1;
         const float* sl = stats + st * 256 + cb;
-        const bool full = !qt.diag && qt.len == kTile && un.tile.len == kTile;
+        const bool full = qt.full;
         wait_bar(bar(kQFullB + st), (g >> 1) & 1, abort_flag, prm.header, 70);
         wait_bar(bar(kSFullB), par, abort_flag, prm.header, 71);
         tc_fence_after();
@@ -442,16 +448,16 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             pk[2 * i + 1] = pack_bf16(p2, p3);
           }
         } else {
-          // visible iff the key row exists, the query column exists, and (diagonal tile) the
-          // query is not before the key
-          const int lo = qt.diag ? row : 0;
+          // query column c is visible iff key_lo <= qt.start + c < key_hi (an absent key row
+          // has an empty range; key_hi never exceeds the group's end, so c < qt.len follows)
+          const int lo = key_lo - qt.start, hi = key_hi - qt.start;
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             const int c0 = cb + 2 * i;
             float p0 = ex2(fmaf(__uint_as_float(v[2 * i]), prm.scale_log2, -sl[2 * i]));
             float p1 = ex2(fmaf(__uint_as_float(v[2 * i + 1]), prm.scale_log2, -sl[2 * i + 1]));
-            p0 = (row_ok && c0 >= lo && c0 < qt.len) ? p0 : 0.f;
-            p1 = (row_ok && c0 + 1 >= lo && c0 + 1 < qt.len) ? p1 : 0.f;
+            p0 = (c0 >= lo && c0 < hi) ? p0 : 0.f;
+            p1 = (c0 + 1 >= lo && c0 + 1 < hi) ? p1 : 0.f;
             pk[i] = pack_bf16(p0, p1);
           }
         }
@@ -715,8 +721,9 @@ cudaError_t launch_bwd(const pp_plan* plan, const void* q, const void* k, const 
   char* sc = static_cast<char*>(scratch);
   BwdParams prm;
   prm.header = reinterpret_cast<int32_t*>(plan->ws + plan->lay.header);
-  prm.tiles = reinterpret_cast<const Tile*>(plan->ws + plan->lay.tiles);
+  prm.tiles = reinterpret_cast<const BTile*>(plan->ws + plan->lay.btiles);
   prm.order = reinterpret_cast<const int32_t*>(plan->ws + plan->lay.bwd_units);
+  prm.key_end = reinterpret_cast<const int32_t*>(plan->ws + plan->lay.key_end);
   prm.delta = reinterpret_cast<float*>(sc + sl.delta);
   prm.lse2 = reinterpret_cast<float*>(sc + sl.lse2);
   prm.dq_acc = reinterpret_cast<float*>(sc + sl.dq_acc);

@@ -24,6 +24,28 @@ struct Tile {
 };
 static_assert(sizeof(Tile) == 32, "tile record is 32 bytes");
 
+// One key tile of the backward pass.  The backward cuts each GROUP (prompt and responses as one
+// token range) into tiles of 128 tokens from the group's start, so a tile may straddle segment
+// boundaries: short segments then leave no ragged tile each, only the group's last tile is
+// short.  Key j of the tile is seen by the queries [j, key_end[j]); the query tiles of the unit
+// are the tiles of the same grid from this one on, up to vis_end.
+struct BTile {
+  int32_t start;      // first token
+  int32_t len;        // 1..128 tokens
+  int32_t vis_end;    // largest key_end of the tile's keys: queries [start, vis_end) see some key
+  int32_t full_end;   // smallest key_end of the tile's keys: queries in [start + len, full_end)
+                      //   see every key of the tile
+  int32_t grp_start;  // first token of the group (also the group's identity)
+  int32_t grp_end;    // one past the last token of the group
+  int32_t work;       // number of query tiles: 1 + ceil((vis_end - start - len) / 128)
+  int32_t pad;
+};
+static_assert(sizeof(BTile) == 32, "backward tile record is 32 bytes");
+
+// Words of the plan header (int32[16]).
+constexpr int kHdrStatus = 0, kHdrDetail = 1, kHdrNumTiles = 2, kHdrNumSegments = 3,
+              kHdrNumBTiles = 8;
+
 // Status word values written by device code.
 enum : int32_t {
   kStatusOk = 0,
@@ -34,16 +56,18 @@ enum : int32_t {
 
 // Device part of a plan: offsets (bytes) into the caller's workspace.
 struct PlanLayout {
-  size_t header;     // int32[8]: status, detail, num_tiles, num_segments, ...
+  size_t header;     // int32[16]: status, detail, num_tiles, num_segments, counters, num_btiles
   size_t desc;       // device copy of the descriptor arrays (when given on host)
   size_t seg_start;  // int32[nseg + 1]
   size_t seg_tile0;  // int32[nseg + 1]  first tile of each segment
   size_t tiles;      // Tile[max_tiles]
   size_t fwd_order;  // int32[max_tiles]
-  size_t bwd_order;  // int32[max_tiles]
-  size_t tile_gwork; // int32[max_tiles]  backward work of the tile's whole group
-  size_t tile_sgroup; // int32[max_tiles] super-group (block of consecutive groups) of the tile
-  size_t bwd_units;  // int32[max_tiles * Hkv]  (kv head << 24) | tile, in processing order
+  size_t grp_btile0; // int32[G + 1]  first backward tile of each group
+  size_t btiles;     // BTile[max_tiles]  (at most T / 128 + G of them)
+  size_t bwd_order;  // int32[max_tiles]  backward tiles, longest work first
+  size_t tile_gwork; // int32[max_tiles]  backward work of the backward tile's whole group
+  size_t tile_sgroup; // int32[max_tiles] super-group (block of consecutive groups)
+  size_t bwd_units;  // int32[max_tiles * Hkv]  (kv head << 24) | backward tile, processing order
   size_t key_end;    // int32[T]
   size_t total;
 };
@@ -82,6 +106,8 @@ inline PlanLayout plan_layout(const pp_problem& p) {
   l.seg_tile0 = off; off = align_up(off + sizeof(int32_t) * (nseg + 1), 256);
   l.tiles = off;     off = align_up(off + sizeof(Tile) * size_t(mt), 256);
   l.fwd_order = off; off = align_up(off + sizeof(int32_t) * size_t(mt), 256);
+  l.grp_btile0 = off; off = align_up(off + sizeof(int32_t) * (size_t(p.num_groups) + 1), 256);
+  l.btiles = off;    off = align_up(off + sizeof(BTile) * size_t(mt), 256);
   l.bwd_order = off; off = align_up(off + sizeof(int32_t) * size_t(mt), 256);
   l.tile_gwork = off; off = align_up(off + sizeof(int32_t) * size_t(mt), 256);
   l.tile_sgroup = off; off = align_up(off + sizeof(int32_t) * size_t(mt), 256);

@@ -4,8 +4,11 @@
 // segment: a key j is seen by the contiguous queries [j, end_j) where end_j is the end of
 // j's group for a prompt key and the end of j's own response otherwise; a query sees at
 // most two contiguous key ranges (its group's prompt, and its own segment up to itself).
-// Tiles are cut per segment (aligned to the segment start), so a tile never straddles two
-// segments and only its own diagonal block needs element-wise causal masking.
+// Forward tiles are cut per segment (aligned to the segment start), so a tile never straddles
+// two segments and only its own diagonal block needs element-wise causal masking.  The
+// backward has its own key tiles, cut per group (see BTile): its masks are two comparisons per
+// element with per-key bounds, so straddling costs nothing there and short segments leave no
+// ragged tiles.
 #include "pp_internal.h"
 
 namespace pp {
@@ -20,6 +23,8 @@ struct PlanPtrs {
   int32_t* seg_start;
   int32_t* seg_tile0;
   Tile* tiles;
+  int32_t* grp_btile0;
+  BTile* btiles;
   int32_t* fwd_order;
   int32_t* bwd_order;
   int32_t* tile_gwork;
@@ -50,7 +55,7 @@ __device__ __forceinline__ bool plan_scan_body(const PlanPtrs& p) {
     p.header[1] = 0;
     p.header[2] = 0;
     p.header[3] = p.nseg;
-    for (int i = 4; i < 8; ++i) p.header[i] = 0;  // dynamic-scheduling counters of the kernels
+    for (int i = 4; i < 16; ++i) p.header[i] = 0;  // [4,8): dynamic-scheduling counters
     if (p.row_group_off[0] != 0 || p.row_group_off[p.num_rows] != p.G)
       set_status(p.header, kStatusBadDescriptor, -1);
     if (p.grp_resp_off[0] != 0 || p.grp_resp_off[p.G] != p.N)
@@ -119,7 +124,38 @@ __device__ __forceinline__ bool plan_scan_body(const PlanPtrs& p) {
     }
   }
   __syncthreads();
-  return p.header[0] == kStatusOk;
+  if (p.header[0] != kStatusOk) return false;
+
+  // backward tiles: ceil(group length / 128) per group, exclusive scan over the groups
+  if (tid == 0) s_carry[1] = 0;
+  __syncthreads();
+  for (int base = 0; base < p.G; base += blockDim.x) {
+    const int g = base + tid;
+    int til = 0;
+    if (g < p.G) {
+      const int gs = p.seg_start[g + p.grp_resp_off[g]];
+      const int ge = p.seg_start[(g + 1) + p.grp_resp_off[g + 1]];
+      til = (ge - gs + kTile - 1) / kTile;
+    }
+    s_til[tid] = til;
+    __syncthreads();
+    for (int d = 1; d < (int)blockDim.x; d <<= 1) {
+      int b = tid >= d ? s_til[tid - d] : 0;
+      __syncthreads();
+      s_til[tid] += b;
+      __syncthreads();
+    }
+    if (g < p.G) p.grp_btile0[g] = s_carry[1] + s_til[tid] - til;
+    __syncthreads();
+    if (tid == blockDim.x - 1) s_carry[1] += s_til[tid];
+    __syncthreads();
+  }
+  if (tid == 0) {
+    p.grp_btile0[p.G] = s_carry[1];
+    p.header[kHdrNumBTiles] = s_carry[1];
+  }
+  __syncthreads();
+  return true;
 }
 
 __global__ void __launch_bounds__(1024) plan_scan_kernel(PlanPtrs p) { plan_scan_body(p); }
@@ -189,30 +225,53 @@ __global__ void plan_key_end_kernel(PlanPtrs p) {
   if (j < p.T) plan_key_end_body(p, j);
 }
 
-__device__ __forceinline__ int bwd_work(const Tile& t) {
-  return 1 + (t.vis_end - (t.start + t.len) + kTile - 1) / kTile;
+// Backward tile t: tile k of its group's 128-token grid.
+__device__ __forceinline__ void plan_btile_body(const PlanPtrs& p, int t) {
+  const int g = upper_segment(p.grp_btile0, p.G, t);
+  const int sp = g + p.grp_resp_off[g];  // the group's prompt segment
+  const int gs = p.seg_start[sp];
+  const int pe = p.seg_start[sp + 1];    // end of the prompt
+  const int ge = p.seg_start[(g + 1) + p.grp_resp_off[g + 1]];
+  BTile b;
+  b.start = gs + (t - p.grp_btile0[g]) * kTile;
+  b.len = min(kTile, ge - b.start);
+  b.grp_start = gs;
+  b.grp_end = ge;
+  // segments of the first and of the last key
+  const int s_first = upper_segment(p.seg_start, p.nseg, b.start);
+  const int s_last = upper_segment(p.seg_start, p.nseg, b.start + b.len - 1);
+  // key_end is the group's end for prompt keys and the own response's end otherwise; along
+  // the tile it is: (group end for the prompt part,) then increasing response ends
+  b.vis_end = (s_first == sp) ? ge : p.seg_start[s_last + 1];
+  if (s_last == sp) b.full_end = ge;                              // prompt keys only
+  else b.full_end = p.seg_start[(s_first == sp ? sp + 1 : s_first) + 1];  // first response part
+  b.work = 1 + (b.vis_end - (b.start + b.len) + kTile - 1) / kTile;
+  b.pad = 0;
+  p.btiles[t] = b;
+}
+
+__global__ void plan_btiles_kernel(PlanPtrs p) {
+  if (p.header[0] != kStatusOk) return;
+  int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t < p.header[kHdrNumBTiles]) plan_btile_body(p, t);
 }
 
 // Longest-work-first orders by rank counting (tile counts are small: T/128 + segments).
-__device__ __forceinline__ void plan_order_body(const PlanPtrs& p, int t, int n) {
-  Tile me = p.tiles[t];
-  int wf = me.work, wb = bwd_work(me);
-  int rf = 0, rb = 0;
+__device__ __forceinline__ void plan_fwd_order_body(const PlanPtrs& p, int t, int n) {
+  const int wf = p.tiles[t].work;
+  int rf = 0;
   for (int u = 0; u < n; ++u) {
-    Tile o = p.tiles[u];
-    int of = o.work, ob = bwd_work(o);
+    const int of = p.tiles[u].work;
     rf += (of > wf) || (of == wf && u < t);
-    rb += (ob > wb) || (ob == wb && u < t);
   }
   p.fwd_order[rf] = t;
-  p.bwd_order[rb] = t;
 }
 
-__global__ void plan_order_kernel(PlanPtrs p) {
+__global__ void plan_fwd_order_kernel(PlanPtrs p) {
   if (p.header[0] != kStatusOk) return;
-  const int n = p.header[2];
+  const int n = p.header[kHdrNumTiles];
   int t = blockIdx.x * blockDim.x + threadIdx.x;
-  if (t < n) plan_order_body(p, t, n);
+  if (t < n) plan_fwd_order_body(p, t, n);
 }
 
 // Backward processing order, built for L2 reuse and balance.  Key tiles of one group stream
@@ -222,24 +281,27 @@ __global__ void plan_order_kernel(PlanPtrs p) {
 // units are ordered longest first (all KV heads of a tile adjacent).  Small problems collapse
 // into one super-group, i.e. a plain longest-first list; large ones keep the working set of the
 // concurrently running units near one group's Q / dO.  Dynamic scheduling in the kernel does
-// the balancing.  A tile's group is identified by the start of its prompt range (kv0_start).
+// the balancing.  A tile's group is identified by the group's first token.
 constexpr int kSuperGroupUnits = 600;
 
+// bwd_order (plain longest-first list of the backward tiles) and each tile's group work
 __device__ __forceinline__ void plan_gwork_body(const PlanPtrs& p, int t, int n) {
-  const int gs = p.tiles[t].kv0_start;
-  int gw = 0;
+  const BTile me = p.btiles[t];
+  int gw = 0, rb = 0;
   for (int u = 0; u < n; ++u) {
-    Tile o = p.tiles[u];
-    gw += (o.kv0_start == gs) ? bwd_work(o) : 0;
+    const BTile o = p.btiles[u];
+    gw += (o.grp_start == me.grp_start) ? o.work : 0;
+    rb += (o.work > me.work) || (o.work == me.work && u < t);
   }
   p.tile_gwork[t] = gw;
+  p.bwd_order[rb] = t;
 }
 
 __device__ __forceinline__ void plan_sgroup_body(const PlanPtrs& p, int t, int n) {
-  const int gs = p.tiles[t].kv0_start, gw = p.tile_gwork[t];
+  const int gs = p.btiles[t].grp_start, gw = p.tile_gwork[t];
   int rest = 0;  // tiles of this group and of the groups that come later
   for (int u = 0; u < n; ++u) {
-    const int ogs = p.tiles[u].kv0_start, ow = p.tile_gwork[u];
+    const int ogs = p.btiles[u].grp_start, ow = p.tile_gwork[u];
     rest += (ogs == gs) || (ow < gw) || (ow == gw && ogs > gs);
   }
   // counted from the END of the list, so the last block is never a small leftover whose
@@ -248,10 +310,10 @@ __device__ __forceinline__ void plan_sgroup_body(const PlanPtrs& p, int t, int n
 }
 
 __device__ __forceinline__ void plan_units_body(const PlanPtrs& p, int t, int n) {
-  const int sg = p.tile_sgroup[t], wb = bwd_work(p.tiles[t]);
+  const int sg = p.tile_sgroup[t], wb = p.btiles[t].work;
   int pos = 0;
   for (int u = 0; u < n; ++u) {
-    const int osg = p.tile_sgroup[u], ob = bwd_work(p.tiles[u]);
+    const int osg = p.tile_sgroup[u], ob = p.btiles[u].work;
     pos += (osg > sg) || (osg == sg && ((ob > wb) || (ob == wb && u < t)));
   }
   for (int kvh = 0; kvh < p.Hkv; ++kvh) p.bwd_units[p.Hkv * pos + kvh] = (kvh << 24) | t;
@@ -259,74 +321,84 @@ __device__ __forceinline__ void plan_units_body(const PlanPtrs& p, int t, int n)
 
 __global__ void plan_gwork_kernel(PlanPtrs p) {
   if (p.header[0] != kStatusOk) return;
-  const int n = p.header[2];
+  const int n = p.header[kHdrNumBTiles];
   int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t < n) plan_gwork_body(p, t, n);
 }
 
 __global__ void plan_sgroup_kernel(PlanPtrs p) {
   if (p.header[0] != kStatusOk) return;
-  const int n = p.header[2];
+  const int n = p.header[kHdrNumBTiles];
   int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t < n) plan_sgroup_body(p, t, n);
 }
 
 __global__ void plan_units_kernel(PlanPtrs p) {
   if (p.header[0] != kStatusOk) return;
-  const int n = p.header[2];
+  const int n = p.header[kHdrNumBTiles];
   int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t < n) plan_units_body(p, t, n);
 }
 
 // The whole plan in one block: used when the problem is small enough that one block's
-// latency beats seven dependent launches (every stage only needs block-level ordering).  The
+// latency beats eight dependent launches (every stage only needs block-level ordering).  The
 // per-tile keys of the rank-counting stages are kept in shared memory, so that the O(n^2)
 // loops do not go through global memory, and key_end is filled tile by tile (every key of a
-// tile ends its visibility at the tile's vis_end) instead of by a search per token.
+// forward tile ends its visibility at the tile's vis_end) instead of by a search per token.
 constexpr int kFusedMaxTiles = 2048;
 
 __global__ void __launch_bounds__(1024) plan_fused_kernel(PlanPtrs p) {
-  __shared__ uint16_t s_wf[kFusedMaxTiles];   // forward work
-  __shared__ uint16_t s_wb[kFusedMaxTiles];   // backward work
-  __shared__ int32_t s_gs[kFusedMaxTiles];    // group id (start of the group's prompt)
+  __shared__ uint16_t s_wf[kFusedMaxTiles];   // forward work of the forward tiles
+  __shared__ uint16_t s_wb[kFusedMaxTiles];   // work of the backward tiles
+  __shared__ int32_t s_gs[kFusedMaxTiles];    // group id of the backward tiles
   __shared__ int32_t s_gw[kFusedMaxTiles];    // backward work of the tile's whole group
   __shared__ uint16_t s_sg[kFusedMaxTiles];   // super-group
   if (!plan_scan_body(p)) return;
-  const int n = p.header[2];
+  const int n = p.header[kHdrNumTiles], nb = p.header[kHdrNumBTiles];
   const int tid = threadIdx.x, nthr = blockDim.x;
   for (int t = tid; t < n; t += nthr) {
     plan_tile_body(p, t);
-    const Tile tl = p.tiles[t];  // own write
-    s_wf[t] = uint16_t(tl.work);
-    s_wb[t] = uint16_t(bwd_work(tl));
-    s_gs[t] = tl.kv0_start;
+    s_wf[t] = uint16_t(p.tiles[t].work);  // own write
+  }
+  for (int t = tid; t < nb; t += nthr) {
+    plan_btile_body(p, t);
+    const BTile b = p.btiles[t];  // own write
+    s_wb[t] = uint16_t(b.work);
+    s_gs[t] = b.grp_start;
   }
   __syncthreads();
-  // key_end: one warp per tile, coalesced
+  // key_end: one warp per forward tile, coalesced
   for (int t = tid >> 5; t < n; t += nthr >> 5) {
     const Tile tl = p.tiles[t];
     for (int i = tid & 31; i < tl.len; i += 32) p.key_end[tl.start + i] = tl.vis_end;
   }
-  // longest-work-first orders by rank counting, and the work of each tile's group
+  // longest-work-first orders by rank counting, and the work of each backward tile's group
   for (int t = tid; t < n; t += nthr) {
-    const int wf = s_wf[t], wb = s_wb[t], gs = s_gs[t];
-    int rf = 0, rb = 0, gw = 0;
+    const int wf = s_wf[t];
+    int rf = 0;
     for (int u = 0; u < n; ++u) {
-      const int of = s_wf[u], ob = s_wb[u];
+      const int of = s_wf[u];
       rf += (of > wf) || (of == wf && u < t);
+    }
+    p.fwd_order[rf] = t;
+  }
+  for (int t = tid; t < nb; t += nthr) {
+    const int wb = s_wb[t], gs = s_gs[t];
+    int rb = 0, gw = 0;
+    for (int u = 0; u < nb; ++u) {
+      const int ob = s_wb[u];
       rb += (ob > wb) || (ob == wb && u < t);
       gw += (s_gs[u] == gs) ? ob : 0;
     }
-    p.fwd_order[rf] = t;
     p.bwd_order[rb] = t;
     p.tile_gwork[t] = gw;
     s_gw[t] = gw;
   }
   __syncthreads();
-  for (int t = tid; t < n; t += nthr) {
+  for (int t = tid; t < nb; t += nthr) {
     const int gs = s_gs[t], gw = s_gw[t];
     int rest = 0;  // tiles of this group and of the groups that come later
-    for (int u = 0; u < n; ++u) {
+    for (int u = 0; u < nb; ++u) {
       const int ogs = s_gs[u], ow = s_gw[u];
       rest += (ogs == gs) || (ow < gw) || (ow == gw && ogs > gs);
     }
@@ -335,10 +407,10 @@ __global__ void __launch_bounds__(1024) plan_fused_kernel(PlanPtrs p) {
     s_sg[t] = uint16_t(sg);
   }
   __syncthreads();
-  for (int t = tid; t < n; t += nthr) {
+  for (int t = tid; t < nb; t += nthr) {
     const int sg = s_sg[t], wb = s_wb[t];
     int pos = 0;
-    for (int u = 0; u < n; ++u) {
+    for (int u = 0; u < nb; ++u) {
       const int osg = s_sg[u], ob = s_wb[u];
       pos += (osg > sg) || (osg == sg && ((ob > wb) || (ob == wb && u < t)));
     }
@@ -390,6 +462,8 @@ cudaError_t launch_plan(const pp_plan* plan, cudaStream_t stream, int* launches)
   p.seg_start = reinterpret_cast<int32_t*>(ws + l.seg_start);
   p.seg_tile0 = reinterpret_cast<int32_t*>(ws + l.seg_tile0);
   p.tiles = reinterpret_cast<Tile*>(ws + l.tiles);
+  p.grp_btile0 = reinterpret_cast<int32_t*>(ws + l.grp_btile0);
+  p.btiles = reinterpret_cast<BTile*>(ws + l.btiles);
   p.fwd_order = reinterpret_cast<int32_t*>(ws + l.fwd_order);
   p.bwd_order = reinterpret_cast<int32_t*>(ws + l.bwd_order);
   p.tile_gwork = reinterpret_cast<int32_t*>(ws + l.tile_gwork);
@@ -413,11 +487,12 @@ cudaError_t launch_plan(const pp_plan* plan, cudaStream_t stream, int* launches)
   plan_scan_kernel<<<1, 1024, 0, stream>>>(p);
   plan_tiles_kernel<<<(mt + 255) / 256, 256, 0, stream>>>(p);
   plan_key_end_kernel<<<(p.T + 255) / 256, 256, 0, stream>>>(p);
-  plan_order_kernel<<<(mt + 127) / 128, 128, 0, stream>>>(p);
+  plan_btiles_kernel<<<(mt + 255) / 256, 256, 0, stream>>>(p);
+  plan_fwd_order_kernel<<<(mt + 127) / 128, 128, 0, stream>>>(p);
   plan_gwork_kernel<<<(mt + 127) / 128, 128, 0, stream>>>(p);
   plan_sgroup_kernel<<<(mt + 127) / 128, 128, 0, stream>>>(p);
   plan_units_kernel<<<(mt + 127) / 128, 128, 0, stream>>>(p);
-  if (launches) *launches = 7;
+  if (launches) *launches = 8;
   return cudaGetLastError();
 }
 

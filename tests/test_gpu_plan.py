@@ -52,7 +52,7 @@ def test_plan_matches_dense_mask(w, desc_on_device):
         want[:, start:start + ln] = np.tril(np.ones((ln, ln), dtype=bool))
         assert np.array_equal(rows, want)
         assert work == (k0l + 127) // 128 + (k1l + 127) // 128 + 1
-        # backward view: the queries that see these keys are exactly [start, vis_end),
+        # column view: the queries that see these keys are exactly [start, vis_end),
         # fully below the tile, causally inside it
         cols = mask[:, start:start + ln]
         wantc = np.zeros((T, ln), dtype=bool)
@@ -60,33 +60,58 @@ def test_plan_matches_dense_mask(w, desc_on_device):
         wantc[start + ln:vis_end] = True
         assert np.array_equal(cols, wantc)
     assert (covered == 1).all()
+    # backward key tiles: every group cut into 128-token tiles from its start
+    btiles = plan.read_bwd_tiles()
+    groups = {}
+    for (s0, l0, _r, g, _k) in segs:
+        lo, hi = groups.get(g, (s0, s0 + l0))
+        groups[g] = (min(lo, s0), max(hi, s0 + l0))
+    assert len(btiles) == sum((hi - lo + 127) // 128 for lo, hi in groups.values())
+    bcov = np.zeros(T, dtype=int)
+    for (start, ln, vis_end, full_end, gstart, gend, work, _pad) in btiles.tolist():
+        assert 1 <= ln <= 128 and (start - gstart) % 128 == 0 and start + ln <= gend
+        assert ln == 128 or start + ln == gend
+        assert (gstart, gend) in groups.values()
+        bcov[start:start + ln] += 1
+        cols = mask[:, start:start + ln]
+        seen = np.nonzero(cols.any(axis=1))[0]
+        assert seen[0] == start and seen[-1] + 1 == vis_end
+        # per-key bounds: key j is seen by exactly [j, key_end[j])
+        for c in range(ln):
+            q = np.nonzero(cols[:, c])[0]
+            assert q[0] == start + c and q[-1] + 1 == key_end[start + c] and len(q) == key_end[start + c] - start - c
+        assert vis_end == key_end[start:start + ln].max() and full_end == key_end[start:start + ln].min()
+        # queries in [start + ln, full_end) see every key of the tile
+        assert cols[start + ln:full_end].all()
+        assert work == 1 + (vis_end - start - ln + 127) // 128
+    assert (bcov == 1).all()
     # column form of the mask: key j is visible to queries [j, key_end[j])
     for j in range(0, T, max(1, T // 997)):
         seen = np.nonzero(mask[:, j])[0]
         assert seen[0] == j and seen[-1] + 1 == key_end[j] and len(seen) == key_end[j] - j
     # orders are permutations, longest work first
-    n = len(tiles)
-    assert sorted(fwd_order.tolist()) == list(range(n)) and sorted(bwd_order.tolist()) == list(range(n))
+    n, nb = len(tiles), len(btiles)
+    bwd_order = bwd_order[:nb]
+    assert sorted(fwd_order.tolist()) == list(range(n)) and sorted(bwd_order.tolist()) == list(range(nb))
     fw = tiles[fwd_order, 7]
     assert (np.diff(fw) <= 0).all()
-    bw = 1 + (tiles[:, 6] - tiles[:, 0] - tiles[:, 1] + 127) // 128
-    assert (np.diff(bw[bwd_order]) <= 0).all()
+    assert (np.diff(btiles[bwd_order, 6]) <= 0).all()
 
 
 @pytest.mark.parametrize("w", CASES + [W.config4(3)], ids=lambda w: w.name)
 def test_backward_units_order(w):
-    """Every (tile, KV head) appears exactly once; groups are taken in order of decreasing
+    """Every (backward tile, KV head) appears exactly once; groups are taken in order of decreasing
     backward work and merged into super-groups of about 600 units; inside a super-group units
     come longest first with all KV heads of a tile adjacent."""
     from paper_2602_24082_b200 import binding as B
     plan = B.plan_for(w, desc_on_device=True)
-    tiles, _, _, _ = plan.read()
-    n, hkv = len(tiles), w.num_kv_heads
+    btiles = plan.read_bwd_tiles()
+    n, hkv = len(btiles), w.num_kv_heads
     units = plan.read_bwd_units(n)
     assert units.shape == (n * hkv, 2)
     assert sorted(map(tuple, units.tolist())) == [(h, t) for h in range(hkv) for t in range(n)]
-    work = 1 + (tiles[:, 6] - tiles[:, 0] - tiles[:, 1] + 127) // 128
-    grp = tiles[:, 2]                      # start of the group's prompt = group identity
+    work = btiles[:, 6]
+    grp = btiles[:, 4]                     # first token of the group = group identity
     gwork = {int(g): int(work[grp == g].sum()) for g in np.unique(grp)}
     ranked = sorted(gwork, key=lambda g: (-gwork[g], g))
     sgroup, rest = {}, n
@@ -108,9 +133,10 @@ def test_multi_kernel_plan_path_matches_fused_semantics():
     plan = B.plan_for(w, desc_on_device=True)
     assert plan.status() == (0, 0)
     tiles, fwd_order, bwd_order, key_end = plan.read()
-    n = len(tiles)
-    assert n == 3 * 1100 and n > 2048
-    assert sorted(fwd_order.tolist()) == list(range(n)) and sorted(bwd_order.tolist()) == list(range(n))
+    btiles = plan.read_bwd_tiles()
+    n, nb = len(tiles), len(btiles)
+    assert n == 3 * 1100 and n > 2048 and nb == 1100     # every group is shorter than a tile
+    assert sorted(fwd_order.tolist()) == list(range(n)) and sorted(bwd_order[:nb].tolist()) == list(range(nb))
     segs = w.segments()
     assert [int(t[0]) for t in tiles] == [s[0] for s in segs] and [int(t[1]) for t in tiles] == [s[1] for s in segs]
     for (start, ln, k0s, k0l, k1s, k1l, vis_end, work), (s0, l0, _, g, seg) in zip(tiles.tolist(), segs):
@@ -120,8 +146,11 @@ def test_multi_kernel_plan_path_matches_fused_semantics():
             assert (k0s, k0l, k1l, vis_end) == (gs[0], 0, 0, gend)
         else:
             assert (k0s, k0l, k1s, k1l, vis_end) == (gs[0], gs[1], s0, 0, s0 + l0)
-    units = plan.read_bwd_units(n)
-    assert sorted(map(tuple, units.tolist())) == [(h, t) for h in range(2) for t in range(n)]
+    units = plan.read_bwd_units(nb)
+    assert sorted(map(tuple, units.tolist())) == [(h, t) for h in range(2) for t in range(nb)]
+    gl = [sum(x[1] for x in segs if x[3] == g) for g in range(1100)]
+    assert btiles[:, 1].tolist() == gl and (btiles[:, 6] == 1).all()
+    assert (btiles[:, 2] == btiles[:, 5]).all()          # prompt keys reach the group's end
     for j in range(0, w.total_tokens, 97):
         seg = [x for x in segs if x[0] <= j < x[0] + x[1]][0]
         gend = max(x[0] + x[1] for x in segs if x[3] == seg[3])
