@@ -62,6 +62,10 @@ RAGGED = [
     ("d128-groups", [[(97, (64, 200)), (128, (128, 128)), (3, (2, 1))]], 2, 2, 128),
     ("d64-gqa4", [[(300, (140, 10, 77, 129))]], 4, 1, 64),
     ("d128-single-response", [[(200, (333,))]], 2, 1, 128),
+    # backward key tiles are cut per group: tiles that hold the prompt's tail and several
+    # whole responses, responses of one token, segment boundaries on and next to tile edges
+    ("d64-many-short-responses", [[(100, (7, 1, 30, 1, 1, 64, 2, 90, 13))]], 2, 1, 64),
+    ("d128-aligned-and-off-by-one", [[(128, (128, 127, 129)), (127, (1, 128)), (129, (130,))]], 2, 2, 128),
 ]
 
 

@@ -11,6 +11,7 @@ CASES = [
     W.config0(),
     W.Workload("ragged", [[(257, (5, 128, 31))], [(1, (1, 300))]], 4, 2, 128, seed=4),
     W.Workload("groups", [[(97, (64, 200)), (128, (128, 128)), (3, (2, 1))], [(700, (1,))]], 2, 2, 64, seed=5),
+    W.Workload("short-responses", [[(100, (7, 1, 30, 1, 1, 64, 2, 90, 13)), (127, (1, 128))]], 2, 1, 64, seed=6),
     W.config3(),
 ]
 
