@@ -228,7 +228,7 @@ def run_ours(args):
         n = B.pp_last_launch_count()
         if "scratch" in plan_holder:
             plan._bwd_scratch = plan_holder["scratch"]
-        B.pp_attn_fwd(plan, q, k, v, scale, o=o, lse=lse)
+        B.pp_attn_fwd(plan, q, k, v, scale, o=o, lse=lse, for_backward=True)
         n += B.pp_last_launch_count()
         B.pp_attn_bwd(plan, q, k, v, o, lse, do, scale, d_q=dq, d_k=dk, d_v=dv)
         n += B.pp_last_launch_count()

@@ -218,7 +218,9 @@ def _chk(t: torch.Tensor, shape, dtype, name):
 
 def pp_attn_fwd(plan: Plan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor,
                 softmax_scale: float, o: Optional[torch.Tensor] = None,
-                lse: Optional[torch.Tensor] = None):
+                lse: Optional[torch.Tensor] = None, for_backward: bool = False):
+    """``for_backward``: also hand the plan's backward scratch to the forward, which then clears
+    the fp32 dQ accumulator in it (the following ``pp_attn_bwd`` skips its own clearing)."""
     p = plan.problem
     T, Hq, Hkv, D = p.total_tokens, p.num_q_heads, p.num_kv_heads, p.head_dim
     _chk(q, (T, Hq, D), torch.bfloat16, "q")
@@ -230,9 +232,13 @@ def pp_attn_fwd(plan: Plan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor,
         lse = torch.empty(Hq, T, dtype=torch.float32, device=q.device)
     _chk(o, (T, Hq, D), torch.bfloat16, "o")
     _chk(lse, (Hq, T), torch.float32, "lse")
+    sc_ptr, sc_bytes = None, 0
+    if for_backward:
+        sc = plan.bwd_scratch()
+        sc_ptr, sc_bytes = sc.data_ptr(), sc.numel()
     with torch.cuda.device(q.device):
         _check(lib().pp_attn_fwd(plan.handle, q.data_ptr(), k.data_ptr(), v.data_ptr(),
-                                 float(softmax_scale), o.data_ptr(), lse.data_ptr(), None, 0,
+                                 float(softmax_scale), o.data_ptr(), lse.data_ptr(), sc_ptr, sc_bytes,
                                  _stream()), "pp_attn_fwd")
     return o, lse
 

@@ -198,15 +198,25 @@ int pp_plan_read(const pp_plan* plan, pp_stream_t stream, int32_t* num_tiles, in
 int pp_attn_fwd(const pp_plan* plan, const void* q, const void* k, const void* v,
                 float softmax_scale, void* o, float* lse, void* d_scratch, size_t scratch_bytes,
                 pp_stream_t stream) {
-  (void)d_scratch;
-  (void)scratch_bytes;
   g_last_launches = 0;
   if (!plan || !q || !k || !v || !o || !lse) return PP_ERR_INVALID_ARG;
   if (!(softmax_scale > 0.f) || softmax_scale > 1e30f) return PP_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse))
     return PP_ERR_ALIGNMENT;
-  cudaError_t e = pp::launch_fwd(plan, q, k, v, softmax_scale, o, lse,
+  // Optional: the buffer the caller will hand to pp_attn_bwd as scratch.  The forward then
+  // also clears the fp32 dQ accumulator inside it (the kernel is compute-bound and has memory
+  // bandwidth to spare), and the backward's preprocess pass skips its own clearing.
+  float* dq_clear = nullptr;
+  plan->cleared_scratch = nullptr;
+  if (d_scratch) {
+    if (scratch_bytes < plan->bwd_scratch) return PP_ERR_WORKSPACE_TOO_SMALL;
+    if (reinterpret_cast<uintptr_t>(d_scratch) & 255) return PP_ERR_ALIGNMENT;
+    dq_clear = reinterpret_cast<float*>(static_cast<char*>(d_scratch) +
+                                        pp::bwd_scratch_layout(plan->prob).dq_acc);
+  }
+  cudaError_t e = pp::launch_fwd(plan, q, k, v, softmax_scale, o, lse, dq_clear,
                                  reinterpret_cast<cudaStream_t>(stream), &g_last_launches);
+  if (e == cudaSuccess && d_scratch) plan->cleared_scratch = d_scratch;
   return e == cudaSuccess ? PP_OK : (e == cudaErrorNotSupported ? PP_ERR_UNSUPPORTED : PP_ERR_CUDA);
 }
 
@@ -222,8 +232,11 @@ int pp_attn_bwd(const pp_plan* plan, const void* q, const void* k, const void* v
   for (const void* p : ptrs)
     if (!aligned16(p)) return PP_ERR_ALIGNMENT;
   if (reinterpret_cast<uintptr_t>(d_scratch) & 255) return PP_ERR_ALIGNMENT;
+  // cleared by the latest forward on this plan (which must precede this call on the stream)?
+  const bool dq_cleared = plan->cleared_scratch == d_scratch;
+  plan->cleared_scratch = nullptr;
   cudaError_t e = pp::launch_bwd(plan, q, k, v, o, lse, d_o, softmax_scale, d_q, d_k, d_v,
-                                 d_scratch, reinterpret_cast<cudaStream_t>(stream),
+                                 d_scratch, dq_cleared, reinterpret_cast<cudaStream_t>(stream),
                                  &g_last_launches);
   return e == cudaSuccess ? PP_OK : (e == cudaErrorNotSupported ? PP_ERR_UNSUPPORTED : PP_ERR_CUDA);
 }
@@ -323,7 +336,8 @@ int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_
   if (rc) return rc;
   int launches = g_last_launches;
   rc = pp_attn_fwd(plan, base + a.q, base + a.k, base + a.v, softmax_scale, base + a.o,
-                   reinterpret_cast<float*>(base + a.lse), nullptr, 0, stream);
+                   reinterpret_cast<float*>(base + a.lse), base + a.scratch, a.total - a.scratch,
+                   stream);
   launches += g_last_launches;
   if (rc == PP_OK) {
     rc = pp_attn_bwd(plan, base + a.q, base + a.k, base + a.v, base + a.o,

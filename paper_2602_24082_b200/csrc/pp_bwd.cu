@@ -37,41 +37,62 @@ struct BwdParams {
 };
 
 // ---------------------------------------------------------------- preprocess
-// One warp per (token, query head) row: Delta = sum_d dO * O, the LSE in base-2 units, and the
-// row of the fp32 dQ accumulator cleared (so no separate memset pass over it is needed).
-template <int D>
+// Delta = sum_d dO * O per (token, query head) row, the LSE in base-2 units, and the row of
+// the fp32 dQ accumulator cleared (so no separate memset pass over it is needed) unless the
+// forward has already cleared it (kClear = false).  D / 8 lanes per row with 16-byte loads,
+// four row groups per warp in flight: the pass is a pure stream over O and dO.
+template <int D, bool kClear>
 __global__ void __launch_bounds__(256)
 bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
                       const float* __restrict__ lse, float* __restrict__ delta,
                       float* __restrict__ lse2, float* __restrict__ dq_acc, int T, int Hq) {
-  const int lane = threadIdx.x & 31;
+  constexpr int kLanes = D / 8;           // lanes per row
+  constexpr int kRows = 32 / kLanes;      // rows per warp and step
+  constexpr int kUnroll = 4;
+  const int lane = threadIdx.x & 31, sub = lane % kLanes, rin = lane / kLanes;
   const long long rows = (long long)T * Hq;
-  const long long stride = (long long)gridDim.x * 8;
-  for (long long idx = (long long)blockIdx.x * 8 + (threadIdx.x >> 5); idx < rows; idx += stride) {
-    const int t = int(idx / Hq), h = int(idx - (long long)t * Hq);
-    float acc = 0.f;
-    if (D == 128) {
-      const uint2 a = reinterpret_cast<const uint2*>(o + idx * D)[lane];
-      const uint2 b = reinterpret_cast<const uint2*>(d_o + idx * D)[lane];
-      const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a.x));
-      const float2 a1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a.y));
-      const float2 b0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b.x));
-      const float2 b1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b.y));
-      acc = a0.x * b0.x + a0.y * b0.y + a1.x * b1.x + a1.y * b1.y;
-      reinterpret_cast<float4*>(dq_acc + idx * D)[lane] = make_float4(0.f, 0.f, 0.f, 0.f);
-    } else {
-      const uint32_t a = reinterpret_cast<const uint32_t*>(o + idx * D)[lane];
-      const uint32_t b = reinterpret_cast<const uint32_t*>(d_o + idx * D)[lane];
-      const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a));
-      const float2 b0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b));
-      acc = a0.x * b0.x + a0.y * b0.y;
-      reinterpret_cast<float2*>(dq_acc + idx * D)[lane] = make_float2(0.f, 0.f);
+  const long long warp0 = ((long long)blockIdx.x * 8 + (threadIdx.x >> 5)) * (kRows * kUnroll);
+  const long long stride = (long long)gridDim.x * 8 * (kRows * kUnroll);
+  for (long long base = warp0; base < rows; base += stride) {
+    uint4 a[kUnroll], b[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      // rows are walked head by head, tokens fastest: the per-row statistics [Hq][T] are then
+      // written to consecutive addresses (each O / dO row is one contiguous piece anyway)
+      const long long idx = base + u * kRows + rin;
+      a[u] = b[u] = make_uint4(0u, 0u, 0u, 0u);
+      if (idx < rows) {
+        const int h = int(idx / T), t = int(idx - (long long)h * T);
+        const long long row = (long long)t * Hq + h;
+        a[u] = reinterpret_cast<const uint4*>(o + row * D)[sub];
+        b[u] = reinterpret_cast<const uint4*>(d_o + row * D)[sub];
+      }
     }
 #pragma unroll
-    for (int sft = 16; sft > 0; sft >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sft);
-    if (lane == 0) {
-      delta[size_t(h) * T + t] = acc;
-      lse2[size_t(h) * T + t] = lse[size_t(h) * T + t] * 1.4426950408889634f;
+    for (int u = 0; u < kUnroll; ++u) {
+      const long long idx = base + u * kRows + rin;
+      const uint32_t aw[4] = {a[u].x, a[u].y, a[u].z, a[u].w}, bw[4] = {b[u].x, b[u].y, b[u].z, b[u].w};
+      float acc = 0.f;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&aw[i]));
+        const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&bw[i]));
+        acc = fmaf(x.x, y.x, fmaf(x.y, y.y, acc));
+      }
+#pragma unroll
+      for (int sft = kLanes / 2; sft > 0; sft >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sft);
+      if (idx < rows) {
+        if (kClear) {
+          const int h = int(idx / T), t = int(idx - (long long)h * T);
+          float4* z = reinterpret_cast<float4*>(dq_acc + ((long long)t * Hq + h) * D + sub * 8);
+          z[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+          z[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        if (sub == 0) {
+          delta[idx] = acc;
+          lse2[idx] = lse[idx] * 1.4426950408889634f;
+        }
+      }
     }
   }
 }
@@ -665,7 +686,8 @@ template <int D>
 cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, const void* d_o,
                          void* dq, const CUtensorMap& tq, const CUtensorMap& tk,
                          const CUtensorMap& tv, const CUtensorMap& tdo, const CUtensorMap& tdq,
-                         const BwdParams& prm, cudaStream_t stream, int* launches) {
+                         const BwdParams& prm, bool dq_cleared, cudaStream_t stream,
+                         int* launches) {
   static bool configured = false;
   auto kern = bwd_kernel<D>;
   if (!configured) {
@@ -677,10 +699,17 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
   const pp_problem& pb = plan->prob;
   const size_t T = pb.total_tokens, Hq = pb.num_q_heads;
   const long long pairs = (long long)T * Hq;
-  const unsigned pre_blocks = unsigned(std::min<long long>((pairs + 7) / 8, 148 * 32));
-  bwd_preprocess_kernel<D><<<pre_blocks, 256, 0, stream>>>(
-      static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse,
-      const_cast<float*>(prm.delta), const_cast<float*>(prm.lse2), prm.dq_acc, int(T), int(Hq));
+  constexpr int kRowsPerBlock = 8 * (32 / (D / 8)) * 4;  // warps x rows per warp x unroll
+  const unsigned pre_blocks =
+      unsigned(std::min<long long>((pairs + kRowsPerBlock - 1) / kRowsPerBlock, 148 * 16));
+  if (dq_cleared)
+    bwd_preprocess_kernel<D, false><<<pre_blocks, 256, 0, stream>>>(
+        static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse,
+        const_cast<float*>(prm.delta), const_cast<float*>(prm.lse2), prm.dq_acc, int(T), int(Hq));
+  else
+    bwd_preprocess_kernel<D, true><<<pre_blocks, 256, 0, stream>>>(
+        static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse,
+        const_cast<float*>(prm.delta), const_cast<float*>(prm.lse2), prm.dq_acc, int(T), int(Hq));
   static int num_sms = 0;
   if (!num_sms) {
     int dev = 0;
@@ -709,7 +738,8 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
 
 cudaError_t launch_bwd(const pp_plan* plan, const void* q, const void* k, const void* v,
                        const void* o, const float* lse, const void* d_o, float scale, void* dq,
-                       void* dk, void* dv, void* scratch, cudaStream_t stream, int* launches) {
+                       void* dk, void* dv, void* scratch, bool dq_cleared, cudaStream_t stream,
+                       int* launches) {
   const pp_problem& pb = plan->prob;
   CUtensorMap tq, tk, tv, tdo;
   if (!encode_thd(&tq, q, pb.total_tokens, pb.num_q_heads, pb.head_dim, kTile) ||
@@ -738,8 +768,10 @@ cudaError_t launch_bwd(const pp_plan* plan, const void* q, const void* k, const 
   if (!encode_thd_f32(&tdq, prm.dq_acc, pb.total_tokens, pb.num_q_heads, pb.head_dim))
     return cudaErrorNotSupported;
   return pb.head_dim == 128
-             ? launch_bwd_t<128>(plan, o, lse, d_o, dq, tq, tk, tv, tdo, tdq, prm, stream, launches)
-             : launch_bwd_t<64>(plan, o, lse, d_o, dq, tq, tk, tv, tdo, tdq, prm, stream, launches);
+             ? launch_bwd_t<128>(plan, o, lse, d_o, dq, tq, tk, tv, tdo, tdq, prm, dq_cleared, stream,
+                                 launches)
+             : launch_bwd_t<64>(plan, o, lse, d_o, dq, tq, tk, tv, tdo, tdq, prm, dq_cleared, stream,
+                                launches);
 }
 
 // ---------------------------------------------------------------- built-in scratch
@@ -778,7 +810,7 @@ cudaError_t launch_bwd_static(const pp_plan* plan, const void* q, const void* k,
   if (e != cudaSuccess) return e;
   // launch_bwd zeroes the fp32 dQ accumulator inside the scratch on every call and rewrites
   // Delta and the scaled LSE, so nothing of an earlier call's contents is read.
-  return launch_bwd(plan, q, k, v, o, lse, d_o, scale, dq, dk, dv, scratch, stream, launches);
+  return launch_bwd(plan, q, k, v, o, lse, d_o, scale, dq, dk, dv, scratch, false, stream, launches);
 }
 
 }  // namespace pp

@@ -9,6 +9,7 @@
 //   warps 2-9   softmax warps of slot 0: two threads per query row (= TMEM lane), 64 key
 //               columns each
 //   warps 10-17 softmax warps of slot 1
+//   warps 18-19 optional: clear the backward's fp32 dQ accumulator for the unit's rows
 // A work unit is (query tile, KV head, pair of query heads of that KV head): both slots see
 // the same keys and the same mask, so every K / V tile staged in shared memory feeds two
 // S tiles.  While one slot's warpgroup does its exponentials the tensor core works on the
@@ -32,11 +33,12 @@ struct FwdParams {
   const int32_t* order;
   __nv_bfloat16* o;
   float* lse;
+  float* dq_clear;  // optional: the backward's fp32 dQ accumulator [T][Hq][D], cleared here
   int T, Hq, Hkv;
   float scale_log2;  // softmax scale * log2(e)
 };
 
-constexpr int kFwdThreads = 576;
+constexpr int kFwdThreads = 640;
 constexpr uint32_t kFwdTmemCols = 512;
 constexpr float kRescaleThreshold = 8.f;  // log2 units
 
@@ -142,7 +144,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     for (int i = 0; i < kNumFwdBars; ++i) {
       const bool wg_count = (i >= kPFull && i < kPFull + 2) || (i >= kOFree && i < kOFree + 2);
       const bool sched_empty = (i >= kSchedEmptyF && i < kSchedEmptyF + 2);
-      mbar_init(bar(i), wg_count ? 256 : (sched_empty ? 17 : 1));
+      // unit records are released by the MMA thread, the 16 softmax warps and, when the dQ
+      // accumulator is cleared here, the two clearing warps
+      mbar_init(bar(i), wg_count ? 256 : (sched_empty ? (prm.dq_clear ? 19 : 17) : 1));
     }
     *abort_flag = 0;
     fence_mbar_init();
@@ -341,6 +345,30 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         }
         ++uc0;
         if (two) ++uc1;
+      }
+    }
+  } else if (warp >= 18) {
+    // ------------------------------------------------------------ clearing warps (optional)
+    // The kernel is compute-bound and leaves most of the memory bandwidth idle: when the
+    // caller passes the backward's scratch, these two warps write zeros over the rows of the
+    // fp32 dQ accumulator that belong to the unit's query tile and heads, so that the
+    // backward needs no clearing pass.  Every (token, query head) row belongs to exactly one
+    // unit and slot.
+    if (prm.dq_clear) {
+      const int cl = (warp - 18) * 32 + lane;  // 0..63
+      for (uint32_t un_i = 0;; ++un_i) {
+        PP_TAKE_UNIT(un_i, true)
+        if (u_nslots == 0) break;
+        constexpr int kChunks = D / 4;  // 16-byte chunks per row
+        const int total = u_len * kChunks;
+        for (int sl = 0; sl < u_nslots; ++sl) {
+          float* base = prm.dq_clear + (size_t(u_start) * prm.Hq + (u_h0 + sl)) * D;
+          for (int c = cl; c < total; c += 64) {
+            const int r = c / kChunks, col = c - r * kChunks;
+            *reinterpret_cast<float4*>(base + size_t(r) * prm.Hq * D + col * 4) =
+                make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+        }
       }
     }
   } else {
@@ -610,7 +638,7 @@ cudaError_t launch_fwd_t(const pp_plan* plan, const CUtensorMap& tq, const CUten
 }  // namespace
 
 cudaError_t launch_fwd(const pp_plan* plan, const void* q, const void* k, const void* v, float scale,
-                       void* o, float* lse, cudaStream_t stream, int* launches) {
+                       void* o, float* lse, float* dq_clear, cudaStream_t stream, int* launches) {
   const pp_problem& pb = plan->prob;
   CUtensorMap tq, tk, tv;
   if (!encode_thd(&tq, q, pb.total_tokens, pb.num_q_heads, pb.head_dim, kTile) ||
@@ -623,6 +651,7 @@ cudaError_t launch_fwd(const pp_plan* plan, const void* q, const void* k, const 
   prm.order = reinterpret_cast<const int32_t*>(plan->ws + plan->lay.fwd_order);
   prm.o = static_cast<__nv_bfloat16*>(o);
   prm.lse = lse;
+  prm.dq_clear = dq_clear;
   prm.T = pb.total_tokens;
   prm.Hq = pb.num_q_heads;
   prm.Hkv = pb.num_kv_heads;

@@ -82,6 +82,8 @@ struct pp_plan {
   pp::PlanLayout lay;
   // scratch sizes
   size_t fwd_scratch, bwd_scratch;
+  // backward scratch whose dQ accumulator the latest forward on this plan has cleared
+  mutable const void* cleared_scratch = nullptr;
 };
 
 namespace pp {
@@ -164,10 +166,11 @@ bool profile_read(float* fwd_ms, float* bwd_ms);
 // launchers (defined in the .cu files); all return a cudaError_t
 cudaError_t launch_plan(const pp_plan* plan, cudaStream_t stream, int* launches);
 cudaError_t launch_fwd(const pp_plan* plan, const void* q, const void* k, const void* v, float scale,
-                       void* o, float* lse, cudaStream_t stream, int* launches);
+                       void* o, float* lse, float* dq_clear, cudaStream_t stream, int* launches);
 cudaError_t launch_bwd(const pp_plan* plan, const void* q, const void* k, const void* v,
                        const void* o, const float* lse, const void* d_o, float scale, void* dq,
-                       void* dk, void* dv, void* scratch, cudaStream_t stream, int* launches);
+                       void* dk, void* dv, void* scratch, bool dq_cleared, cudaStream_t stream,
+                       int* launches);
 
 // Size of the scratch array built into the library image for pp_attn_bwd_noalloc.
 constexpr size_t kStaticScratchBytes = size_t(32) << 20;

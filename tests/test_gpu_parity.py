@@ -16,11 +16,16 @@ pytestmark = pytest.mark.gpu
 TOL_O, TOL_LSE, TOL_GRAD = 2e-2, 5e-3, 2e-2
 
 
-def _run_gpu(w, tens, desc_on_device=False):
+def _run_gpu(w, tens, desc_on_device=False, for_backward=False):
+    """``for_backward``: the forward gets the backward's scratch and clears the dQ accumulator
+    in it (the path the benchmark times); the scratch is filled with NaN bit patterns first, so
+    a row the forward failed to clear would show."""
     from paper_2602_24082_b200 import binding as B
     q, k, v, do = (x.cuda() for x in tens)
     plan = B.plan_for(w, desc_on_device=desc_on_device)
-    o, lse = B.pp_attn_fwd(plan, q, k, v, w.softmax_scale)
+    if for_backward:
+        plan.bwd_scratch().fill_(0xFF)
+    o, lse = B.pp_attn_fwd(plan, q, k, v, w.softmax_scale, for_backward=for_backward)
     dq, dk, dv = B.pp_attn_bwd(plan, q, k, v, o, lse, do, w.softmax_scale)
     torch.cuda.synchronize()
     assert plan.status() == (0, 0)
@@ -74,7 +79,7 @@ RAGGED = [
 def test_ragged_shapes(name, rows, hq, hkv, d, desc_on_device):
     w = W.Workload(name, rows, hq, hkv, d, seed=100 + len(name))
     tens = w.tensors()
-    check_against_oracle(w, tens, _run_gpu(w, tens, desc_on_device))
+    check_against_oracle(w, tens, _run_gpu(w, tens, desc_on_device, for_backward=desc_on_device))
 
 
 def _subset_parity(w, row_ids, kv_heads):
@@ -97,7 +102,8 @@ def _group_parity(w, groups, kv_heads):
     tens = w.tensors()
     q, k, v, do = (x.cuda() for x in tens)
     plan = B.plan_for(w, desc_on_device=True)
-    o, lse = B.pp_attn_fwd(plan, q, k, v, w.softmax_scale)
+    plan.bwd_scratch().fill_(0xFF)
+    o, lse = B.pp_attn_fwd(plan, q, k, v, w.softmax_scale, for_backward=True)
     dq, dk, dv = B.pp_attn_bwd(plan, q, k, v, o, lse, do, w.softmax_scale)
     torch.cuda.synchronize()
     assert plan.status() == (0, 0)
@@ -177,6 +183,29 @@ def test_deterministic_forward_and_dkdv():
     for i in (0, 1, 3, 4):
         assert np.array_equal(a[i], b[i])
     assert _rel_l2(a[2], b[2]) < 1e-3
+
+
+def test_backward_clears_its_accumulator_when_the_forward_did_not():
+    """One forward that cleared the accumulator, then TWO backward calls: the first skips its
+    clearing pass, the second must clear for itself (the accumulator now holds the first
+    call's sums); a forward without the scratch in between resets the hand-over as well."""
+    from paper_2602_24082_b200 import binding as B
+    w = W.Workload("clear", [[(150, (70, 200))], [(40, (129,))]], 4, 2, 128, seed=11)
+    q, k, v, do = (x.cuda() for x in w.tensors())
+    plan = B.plan_for(w)
+    plan.bwd_scratch().fill_(0xFF)
+    o, lse = B.pp_attn_fwd(plan, q, k, v, w.softmax_scale, for_backward=True)
+    a = [x.clone() for x in B.pp_attn_bwd(plan, q, k, v, o, lse, do, w.softmax_scale)]
+    b = [x.clone() for x in B.pp_attn_bwd(plan, q, k, v, o, lse, do, w.softmax_scale)]
+    B.pp_attn_fwd(plan, q, k, v, w.softmax_scale, for_backward=True)
+    B.pp_attn_fwd(plan, q, k, v, w.softmax_scale)          # cancels the hand-over
+    c = [x.clone() for x in B.pp_attn_bwd(plan, q, k, v, o, lse, do, w.softmax_scale)]
+    torch.cuda.synchronize()
+    for x, y, z in zip(a, b, c):
+        assert bool(torch.isfinite(x.float()).all())
+        for other in (y, z):
+            d = (x.float() - other.float()).norm() / x.float().norm()
+            assert float(d) < 1e-3
 
 
 def test_outputs_outside_tiles_untouched():
