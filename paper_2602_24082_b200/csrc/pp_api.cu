@@ -206,17 +206,23 @@ int pp_attn_fwd(const pp_plan* plan, const void* q, const void* k, const void* v
   // Optional: the buffer the caller will hand to pp_attn_bwd as scratch.  The forward then
   // also clears the fp32 dQ accumulator inside it (the kernel is compute-bound and has memory
   // bandwidth to spare), and the backward's preprocess pass skips its own clearing.
+  // Measured: it pays while the accumulator is a few hundred MB (0.15-0.3 GB: step -4..5 %);
+  // at 1 GB the extra stores slow the forward's loads and the zeros have left L2 long before
+  // the backward adds to them (step +2 %), so larger accumulators are left to the backward.
+  constexpr size_t kFwdClearMaxBytes = size_t(320) << 20;
   float* dq_clear = nullptr;
   plan->cleared_scratch = nullptr;
   if (d_scratch) {
     if (scratch_bytes < plan->bwd_scratch) return PP_ERR_WORKSPACE_TOO_SMALL;
     if (reinterpret_cast<uintptr_t>(d_scratch) & 255) return PP_ERR_ALIGNMENT;
-    dq_clear = reinterpret_cast<float*>(static_cast<char*>(d_scratch) +
-                                        pp::bwd_scratch_layout(plan->prob).dq_acc);
+    const pp_problem& pb = plan->prob;
+    if (size_t(4) * pb.total_tokens * pb.num_q_heads * pb.head_dim <= kFwdClearMaxBytes)
+      dq_clear = reinterpret_cast<float*>(static_cast<char*>(d_scratch) +
+                                          pp::bwd_scratch_layout(pb).dq_acc);
   }
   cudaError_t e = pp::launch_fwd(plan, q, k, v, softmax_scale, o, lse, dq_clear,
                                  reinterpret_cast<cudaStream_t>(stream), &g_last_launches);
-  if (e == cudaSuccess && d_scratch) plan->cleared_scratch = d_scratch;
+  if (e == cudaSuccess && dq_clear) plan->cleared_scratch = d_scratch;
   return e == cudaSuccess ? PP_OK : (e == cudaErrorNotSupported ? PP_ERR_UNSUPPORTED : PP_ERR_CUDA);
 }
 
