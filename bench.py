@@ -389,6 +389,25 @@ def run_ours(args):
                                                  "peak": hbm, "unit": "GB/s",
                                                  "frac": lbytes / (statistics.median(lms) * 1e-3) / 1e9 / hbm}}
 
+        # ---- next row: the bit-reproducible backward (key tiles add to dQ in turn)
+        dplan = plan_holder["plan"]
+        B.pp_profile_enable(True)
+        B.pp_attn_fwd(dplan, q, k, v, scale, o=o, lse=lse)   # (both event pairs must be valid)
+        dms, nms = [], []
+        for det in (True, False, True, False):
+            for _ in range(6):
+                flush.zero_()
+                B.pp_attn_bwd(dplan, q, k, v, o, lse, do, scale, d_q=dq, d_k=dk, d_v=dv,
+                              deterministic=det)
+                torch.cuda.synchronize()
+                (dms if det else nms).append(B.pp_profile_read()[1])
+        B.pp_profile_enable(False)
+        bflops = 10.0 * Hq * D * w.useful_pairs()
+        extra["deterministic_bwd"] = {
+            "main_kernel_ms": statistics.median(dms), "default_main_kernel_ms": statistics.median(nms),
+            "tflops": bflops / (statistics.median(dms) * 1e-3) / 1e12,
+            "slowdown": statistics.median(dms) / statistics.median(nms)}
+
     # ---- the CPU oracle beside it (rank 0, N = 1 only), on a bounded sample
     cpu = None
     if world == 1 and not args.no_cpu_baseline:

@@ -25,7 +25,7 @@ EXPORTS = ["pp_plan_workspace_bytes", "pp_build_plan", "pp_plan_status", "pp_des
            "pp_last_launch_count", "pp_error_string", "pp_step_host_arena_bytes",
            "pp_attn_step_host", "pp_profile_enable", "pp_profile_read",
            "pp_attn_bwd_noalloc", "pp_attn_bwd_noalloc_max_bytes", "pp_plan_read_bwd_units",
-           "pp_plan_read_bwd_tiles",
+           "pp_plan_read_bwd_tiles", "pp_attn_bwd_deterministic",
            "pp_position_ids", "pp_rope_qk", "pp_preference_loss"]
 
 
@@ -72,6 +72,7 @@ def lib() -> ctypes.CDLL:
         L.pp_plan_read.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         L.pp_attn_fwd.argtypes = [vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, sz, vp]
         L.pp_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, sz, vp]
+        L.pp_attn_bwd_deterministic.argtypes = L.pp_attn_bwd.argtypes
         L.pp_step_host_arena_bytes.argtypes = [vp, vp]
         L.pp_attn_step_host.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp, sz, vp]
         L.pp_attn_bwd_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
@@ -133,7 +134,7 @@ class Plan:
         return tiles[:n.value], fo[:n.value], bo[:n.value], ke
 
     def read_bwd_tiles(self) -> np.ndarray:
-        """Backward key tiles [n, 8]: start, len, vis_end, full_end, grp_start, grp_end, work, 0."""
+        """Backward key tiles [n, 8]: start, len, vis_end, full_end, grp_start, grp_end, work, npc."""
         mt = lib().pp_plan_max_tiles(self.handle)
         bt = np.zeros((mt, 8), dtype=np.int32)
         n = ctypes.c_int32(0)
@@ -243,7 +244,9 @@ def pp_attn_fwd(plan: Plan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor,
     return o, lse
 
 
-def pp_attn_bwd(plan: Plan, q, k, v, o, lse, d_o, softmax_scale: float, d_q=None, d_k=None, d_v=None):
+def pp_attn_bwd(plan: Plan, q, k, v, o, lse, d_o, softmax_scale: float, d_q=None, d_k=None, d_v=None,
+                deterministic: bool = False):
+    """``deterministic``: pp_attn_bwd_deterministic (bit-reproducible dQ; key tiles take turns)."""
     p = plan.problem
     T, Hq, Hkv, D = p.total_tokens, p.num_q_heads, p.num_kv_heads, p.head_dim
     _chk(q, (T, Hq, D), torch.bfloat16, "q")
@@ -256,11 +259,12 @@ def pp_attn_bwd(plan: Plan, q, k, v, o, lse, d_o, softmax_scale: float, d_q=None
     d_k = torch.empty_like(k) if d_k is None else d_k
     d_v = torch.empty_like(v) if d_v is None else d_v
     scratch = plan.bwd_scratch()
+    fn = lib().pp_attn_bwd_deterministic if deterministic else lib().pp_attn_bwd
     with torch.cuda.device(q.device):
-        _check(lib().pp_attn_bwd(plan.handle, q.data_ptr(), k.data_ptr(), v.data_ptr(),
-                                 o.data_ptr(), lse.data_ptr(), d_o.data_ptr(), float(softmax_scale),
-                                 d_q.data_ptr(), d_k.data_ptr(), d_v.data_ptr(), scratch.data_ptr(),
-                                 scratch.numel(), _stream()), "pp_attn_bwd")
+        _check(fn(plan.handle, q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                  o.data_ptr(), lse.data_ptr(), d_o.data_ptr(), float(softmax_scale),
+                  d_q.data_ptr(), d_k.data_ptr(), d_v.data_ptr(), scratch.data_ptr(),
+                  scratch.numel(), _stream()), "pp_attn_bwd")
     return d_q, d_k, d_v
 
 

@@ -226,9 +226,10 @@ int pp_attn_fwd(const pp_plan* plan, const void* q, const void* k, const void* v
   return e == cudaSuccess ? PP_OK : (e == cudaErrorNotSupported ? PP_ERR_UNSUPPORTED : PP_ERR_CUDA);
 }
 
-int pp_attn_bwd(const pp_plan* plan, const void* q, const void* k, const void* v, const void* o,
-                const float* lse, const void* d_o, float softmax_scale, void* d_q, void* d_k,
-                void* d_v, void* d_scratch, size_t scratch_bytes, pp_stream_t stream) {
+static int attn_bwd_common(const pp_plan* plan, const void* q, const void* k, const void* v,
+                           const void* o, const float* lse, const void* d_o, float softmax_scale,
+                           void* d_q, void* d_k, void* d_v, void* d_scratch, size_t scratch_bytes,
+                           pp_stream_t stream, bool deterministic) {
   g_last_launches = 0;
   if (!plan || !q || !k || !v || !o || !lse || !d_o || !d_q || !d_k || !d_v || !d_scratch)
     return PP_ERR_INVALID_ARG;
@@ -242,9 +243,24 @@ int pp_attn_bwd(const pp_plan* plan, const void* q, const void* k, const void* v
   const bool dq_cleared = plan->cleared_scratch == d_scratch;
   plan->cleared_scratch = nullptr;
   cudaError_t e = pp::launch_bwd(plan, q, k, v, o, lse, d_o, softmax_scale, d_q, d_k, d_v,
-                                 d_scratch, dq_cleared, reinterpret_cast<cudaStream_t>(stream),
-                                 &g_last_launches);
+                                 d_scratch, dq_cleared, deterministic,
+                                 reinterpret_cast<cudaStream_t>(stream), &g_last_launches);
   return e == cudaSuccess ? PP_OK : (e == cudaErrorNotSupported ? PP_ERR_UNSUPPORTED : PP_ERR_CUDA);
+}
+
+int pp_attn_bwd(const pp_plan* plan, const void* q, const void* k, const void* v, const void* o,
+                const float* lse, const void* d_o, float softmax_scale, void* d_q, void* d_k,
+                void* d_v, void* d_scratch, size_t scratch_bytes, pp_stream_t stream) {
+  return attn_bwd_common(plan, q, k, v, o, lse, d_o, softmax_scale, d_q, d_k, d_v, d_scratch,
+                         scratch_bytes, stream, false);
+}
+
+int pp_attn_bwd_deterministic(const pp_plan* plan, const void* q, const void* k, const void* v,
+                              const void* o, const float* lse, const void* d_o,
+                              float softmax_scale, void* d_q, void* d_k, void* d_v,
+                              void* d_scratch, size_t scratch_bytes, pp_stream_t stream) {
+  return attn_bwd_common(plan, q, k, v, o, lse, d_o, softmax_scale, d_q, d_k, d_v, d_scratch,
+                         scratch_bytes, stream, true);
 }
 
 int pp_attn_bwd_noalloc_max_bytes(size_t* bytes) {

@@ -30,6 +30,7 @@ struct BwdParams {
   const float* delta;  // [Hq][T]
   const float* lse2;   // [Hq][T]  LSE * log2(e)
   float* dq_acc;       // [T][Hq][D] fp32
+  int32_t* dq_sem;     // deterministic variant: turn counters [backward tile][Hq]; else null
   __nv_bfloat16* dk;
   __nv_bfloat16* dv;
   int T, Hq, Hkv;
@@ -166,7 +167,7 @@ struct BwdSmem {
 
 struct BwdUnit {
   BTile tile;
-  int kvh, nq, n_it;
+  int kvh, nq, n_it, tidx;
 };
 
 // Units are handed out dynamically: the producer warp draws the next index of the plan's
@@ -181,7 +182,8 @@ __device__ __forceinline__ bool get_bwd_unit(const BwdParams& prm, int u, int nt
   if (u < 0 || u >= ntiles_total * prm.Hkv) return false;
   const int packed = prm.order[u];  // (kv head << 24) | backward tile
   un.kvh = packed >> 24;
-  un.tile = prm.tiles[packed & 0xffffff];
+  un.tidx = packed & 0xffffff;
+  un.tile = prm.tiles[un.tidx];
   un.nq = un.tile.work;
   un.n_it = un.nq * (prm.Hq / prm.Hkv);
   return true;
@@ -605,9 +607,21 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     BwdUnit un;
     for (; get_bwd_unit(prm, take_unit(ucnt, true), ntiles_total, un); ++ucnt) {
       QIter qi;
+      // Deterministic variant: the key tiles that add to a (query tile, head) do so in
+      // ascending tile order.  The counter of the pair holds 1 + the group-relative index of
+      // the last key tile that has added (0: none yet); this unit's turn comes when it shows
+      // the previous contributor -- the tile before this one if that tile reaches the query
+      // tile, else the group's last tile with prompt keys.  In this variant units are handed
+      // out in ascending tile order within a group (the plan's second unit list), so the tile
+      // waited for is always running or done and the waits cannot lock up.
+      const int k_rel = (un.tile.start - un.tile.grp_start) / kTile;
+      int prev_vis_end = 0;
+      if (prm.dq_sem && leader && k_rel > 0) prev_vis_end = prm.tiles[un.tidx - 1].vis_end;
       for (int it = 0; it < un.n_it; ++it, q_advance(qi, prm.Hq / prm.Hkv)) {
         const QTile qt = q_tile_at(prm, un, qi);
         const uint32_t g = gc + it;
+        int32_t* sem = nullptr;
+        if (prm.dq_sem && leader) sem = prm.dq_sem + size_t(un.tidx + qi.qt) * prm.Hq + qt.h;
         wait_bar(bar(kDqFull), g & 1, abort_flag, prm.header, 80);
         tc_fence_after();
         // Two halves of D/2 columns.  The second half is read out of tensor memory (and the
@@ -647,10 +661,36 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             fence_proxy_async_smem();
             named_barrier_sync(1, 128);
             if (leader) {
+              if (sem && half == 0 && c == 0) {  // wait for this unit's turn (bounded)
+                const int expect =
+                    k_rel == 0 ? 0 : (prev_vis_end > qt.start ? k_rel : un.tile.npc);
+                bool ok = false;
+                for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
+                  int seen;
+                  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(sem) : "memory");
+                  if (seen == expect) {
+                    ok = true;
+                    break;
+                  }
+                  if ((spin & 0xff) == 0xff && *abort_flag) break;
+                  __nanosleep(20);
+                }
+                if (!ok && !*abort_flag) {
+                  if (atomicCAS(&prm.header[0], kStatusOk, kStatusWaitExpired) == kStatusOk)
+                    prm.header[1] = 81;
+                  *abort_flag = 1;
+                }
+              }
               tma_reduce_add_3d(&tm_dq, buf, half * (D / 2) + c * 32, qt.h, qt.start);
               bulk_commit_group();
             }
           }
+        }
+        if (sem) {  // all four boxes of the tile added and visible: pass the turn on
+          bulk_wait_group<0>();
+          __threadfence();
+          const int mine = k_rel + 1;
+          asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(sem), "r"(mine) : "memory");
         }
       }
       gc += un.n_it;
@@ -749,8 +789,8 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
 
 cudaError_t launch_bwd(const pp_plan* plan, const void* q, const void* k, const void* v,
                        const void* o, const float* lse, const void* d_o, float scale, void* dq,
-                       void* dk, void* dv, void* scratch, bool dq_cleared, cudaStream_t stream,
-                       int* launches) {
+                       void* dk, void* dv, void* scratch, bool dq_cleared, bool deterministic,
+                       cudaStream_t stream, int* launches) {
   const pp_problem& pb = plan->prob;
   CUtensorMap tq, tk, tv, tdo;
   if (!encode_thd(&tq, q, pb.total_tokens, pb.num_q_heads, pb.head_dim, kTile) ||
@@ -763,11 +803,18 @@ cudaError_t launch_bwd(const pp_plan* plan, const void* q, const void* k, const 
   BwdParams prm;
   prm.header = reinterpret_cast<int32_t*>(plan->ws + plan->lay.header);
   prm.tiles = reinterpret_cast<const BTile*>(plan->ws + plan->lay.btiles);
-  prm.order = reinterpret_cast<const int32_t*>(plan->ws + plan->lay.bwd_units);
+  prm.order = reinterpret_cast<const int32_t*>(
+      plan->ws + (deterministic ? plan->lay.bwd_units_det : plan->lay.bwd_units));
   prm.key_end = reinterpret_cast<const int32_t*>(plan->ws + plan->lay.key_end);
   prm.delta = reinterpret_cast<float*>(sc + sl.delta);
   prm.lse2 = reinterpret_cast<float*>(sc + sl.lse2);
   prm.dq_acc = reinterpret_cast<float*>(sc + sl.dq_acc);
+  prm.dq_sem = nullptr;
+  if (deterministic) {
+    prm.dq_sem = reinterpret_cast<int32_t*>(sc + sl.sem);
+    cudaError_t me = cudaMemsetAsync(prm.dq_sem, 0, sl.sem_bytes, stream);
+    if (me != cudaSuccess) return me;
+  }
   prm.dk = static_cast<__nv_bfloat16*>(dk);
   prm.dv = static_cast<__nv_bfloat16*>(dv);
   prm.T = pb.total_tokens;
@@ -821,7 +868,8 @@ cudaError_t launch_bwd_static(const pp_plan* plan, const void* q, const void* k,
   if (e != cudaSuccess) return e;
   // launch_bwd zeroes the fp32 dQ accumulator inside the scratch on every call and rewrites
   // Delta and the scaled LSE, so nothing of an earlier call's contents is read.
-  return launch_bwd(plan, q, k, v, o, lse, d_o, scale, dq, dk, dv, scratch, false, stream, launches);
+  return launch_bwd(plan, q, k, v, o, lse, d_o, scale, dq, dk, dv, scratch, false, false, stream,
+                    launches);
 }
 
 }  // namespace pp

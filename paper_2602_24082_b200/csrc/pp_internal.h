@@ -38,7 +38,7 @@ struct BTile {
   int32_t grp_start;  // first token of the group (also the group's identity)
   int32_t grp_end;    // one past the last token of the group
   int32_t work;       // number of query tiles: 1 + ceil((vis_end - start - len) / 128)
-  int32_t pad;
+  int32_t npc;        // tiles of the group that hold prompt keys: ceil(prompt length / 128)
 };
 static_assert(sizeof(BTile) == 32, "backward tile record is 32 bytes");
 
@@ -68,6 +68,8 @@ struct PlanLayout {
   size_t tile_gwork; // int32[max_tiles]  backward work of the backward tile's whole group
   size_t tile_sgroup; // int32[max_tiles] super-group (block of consecutive groups)
   size_t bwd_units;  // int32[max_tiles * Hkv]  (kv head << 24) | backward tile, processing order
+  size_t bwd_units_det;  // the same units, inside a super-group by ascending tile index: the
+                         //   order of the deterministic backward
   size_t key_end;    // int32[T]
   size_t total;
 };
@@ -114,14 +116,18 @@ inline PlanLayout plan_layout(const pp_problem& p) {
   l.tile_gwork = off; off = align_up(off + sizeof(int32_t) * size_t(mt), 256);
   l.tile_sgroup = off; off = align_up(off + sizeof(int32_t) * size_t(mt), 256);
   l.bwd_units = off; off = align_up(off + sizeof(int32_t) * size_t(mt) * size_t(p.num_kv_heads), 256);
+  l.bwd_units_det = off;
+  off = align_up(off + sizeof(int32_t) * size_t(mt) * size_t(p.num_kv_heads), 256);
   l.key_end = off;   off = align_up(off + sizeof(int32_t) * size_t(p.total_tokens), 256);
   l.total = off;
   return l;
 }
 
-// Backward scratch: fp32 dQ accumulator [T][Hq][D], Delta [Hq][T], LSE*log2(e) [Hq][T]
+// Backward scratch: fp32 dQ accumulator [T][Hq][D], Delta [Hq][T], LSE*log2(e) [Hq][T], and
+// the turn counters of the deterministic variant, one per (query tile of the backward grid,
+// query head)
 struct BwdScratch {
-  size_t dq_acc, delta, lse2, total;
+  size_t dq_acc, delta, lse2, sem, sem_bytes, total;
 };
 inline BwdScratch bwd_scratch_layout(const pp_problem& p) {
   BwdScratch s{};
@@ -130,6 +136,9 @@ inline BwdScratch bwd_scratch_layout(const pp_problem& p) {
   s.dq_acc = off; off = align_up(off + 4 * T * Hq * D, 256);
   s.delta = off;  off = align_up(off + 4 * T * Hq, 256);
   s.lse2 = off;   off = align_up(off + 4 * T * Hq, 256);
+  s.sem = off;
+  s.sem_bytes = 4 * size_t(max_tiles_of(p)) * Hq;
+  off = align_up(off + s.sem_bytes, 256);
   s.total = off;
   return s;
 }
@@ -169,8 +178,8 @@ cudaError_t launch_fwd(const pp_plan* plan, const void* q, const void* k, const 
                        void* o, float* lse, float* dq_clear, cudaStream_t stream, int* launches);
 cudaError_t launch_bwd(const pp_plan* plan, const void* q, const void* k, const void* v,
                        const void* o, const float* lse, const void* d_o, float scale, void* dq,
-                       void* dk, void* dv, void* scratch, bool dq_cleared, cudaStream_t stream,
-                       int* launches);
+                       void* dk, void* dv, void* scratch, bool dq_cleared, bool deterministic,
+                       cudaStream_t stream, int* launches);
 
 // Size of the scratch array built into the library image for pp_attn_bwd_noalloc.
 constexpr size_t kStaticScratchBytes = size_t(32) << 20;

@@ -30,6 +30,7 @@ struct PlanPtrs {
   int32_t* tile_gwork;
   int32_t* tile_sgroup;
   int32_t* bwd_units;
+  int32_t* bwd_units_det;
   int Hkv;
   int32_t* key_end;
   int num_rows, G, N, T, nseg, max_tiles;
@@ -246,7 +247,7 @@ __device__ __forceinline__ void plan_btile_body(const PlanPtrs& p, int t) {
   if (s_last == sp) b.full_end = ge;                              // prompt keys only
   else b.full_end = p.seg_start[(s_first == sp ? sp + 1 : s_first) + 1];  // first response part
   b.work = 1 + (b.vis_end - (b.start + b.len) + kTile - 1) / kTile;
-  b.pad = 0;
+  b.npc = (pe - gs + kTile - 1) / kTile;
   p.btiles[t] = b;
 }
 
@@ -317,6 +318,14 @@ __device__ __forceinline__ void plan_units_body(const PlanPtrs& p, int t, int n)
     pos += (osg > sg) || (osg == sg && ((ob > wb) || (ob == wb && u < t)));
   }
   for (int kvh = 0; kvh < p.Hkv; ++kvh) p.bwd_units[p.Hkv * pos + kvh] = (kvh << 24) | t;
+  // deterministic order: inside a super-group by ascending tile index, so that every tile of
+  // a group is handed out after the group's earlier tiles
+  int dpos = 0;
+  for (int u = 0; u < n; ++u) {
+    const int osg = p.tile_sgroup[u];
+    dpos += (osg > sg) || (osg == sg && u < t);
+  }
+  for (int kvh = 0; kvh < p.Hkv; ++kvh) p.bwd_units_det[p.Hkv * dpos + kvh] = (kvh << 24) | t;
 }
 
 __global__ void plan_gwork_kernel(PlanPtrs p) {
@@ -409,12 +418,16 @@ __global__ void __launch_bounds__(1024) plan_fused_kernel(PlanPtrs p) {
   __syncthreads();
   for (int t = tid; t < nb; t += nthr) {
     const int sg = s_sg[t], wb = s_wb[t];
-    int pos = 0;
+    int pos = 0, dpos = 0;
     for (int u = 0; u < nb; ++u) {
       const int osg = s_sg[u], ob = s_wb[u];
       pos += (osg > sg) || (osg == sg && ((ob > wb) || (ob == wb && u < t)));
+      dpos += (osg > sg) || (osg == sg && u < t);
     }
-    for (int kvh = 0; kvh < p.Hkv; ++kvh) p.bwd_units[p.Hkv * pos + kvh] = (kvh << 24) | t;
+    for (int kvh = 0; kvh < p.Hkv; ++kvh) {
+      p.bwd_units[p.Hkv * pos + kvh] = (kvh << 24) | t;
+      p.bwd_units_det[p.Hkv * dpos + kvh] = (kvh << 24) | t;  // ascending tiles in a super-group
+    }
   }
 }
 
@@ -469,6 +482,7 @@ cudaError_t launch_plan(const pp_plan* plan, cudaStream_t stream, int* launches)
   p.tile_gwork = reinterpret_cast<int32_t*>(ws + l.tile_gwork);
   p.tile_sgroup = reinterpret_cast<int32_t*>(ws + l.tile_sgroup);
   p.bwd_units = reinterpret_cast<int32_t*>(ws + l.bwd_units);
+  p.bwd_units_det = reinterpret_cast<int32_t*>(ws + l.bwd_units_det);
   p.Hkv = plan->prob.num_kv_heads;
   p.key_end = reinterpret_cast<int32_t*>(ws + l.key_end);
   p.num_rows = plan->prob.num_rows;

@@ -185,6 +185,57 @@ def test_deterministic_forward_and_dkdv():
     assert _rel_l2(a[2], b[2]) < 1e-3
 
 
+DET_CASES = [
+    ("short", [[(300, (140, 77))], [(64, (200, 1))]], 4, 2, 128),
+    # a long response starting inside a tile that also holds the tail of a short one, several
+    # groups, tiles that straddle segments: the turn order has to follow the tile order
+    ("inversions", [[(200, (150, 40, 900)), (127, (1, 128)), (513, (3, 700, 2))]], 4, 2, 64),
+    ("many-heads", [[(1000, (300, 500))], [(129, (640,))]], 8, 2, 128),
+]
+
+
+@pytest.mark.parametrize("name,rows,hq,hkv,d", DET_CASES, ids=[c[0] for c in DET_CASES])
+def test_deterministic_backward(name, rows, hq, hkv, d):
+    """pp_attn_bwd_deterministic: dQ (and everything else) bit-identical between runs, and the
+    same parity with the oracle as the default backward."""
+    from paper_2602_24082_b200 import binding as B
+    w = W.Workload("det-" + name, rows, hq, hkv, d, seed=21)
+    tens = w.tensors()
+    q, k, v, do = (x.cuda() for x in tens)
+    plan = B.plan_for(w)
+    o, lse = B.pp_attn_fwd(plan, q, k, v, w.softmax_scale)
+    runs = []
+    for _ in range(3):
+        plan.bwd_scratch().fill_(0xFF)
+        runs.append([x.clone() for x in B.pp_attn_bwd(plan, q, k, v, o, lse, do, w.softmax_scale,
+                                                      deterministic=True)])
+    torch.cuda.synchronize()
+    assert plan.status() == (0, 0)
+    for r in runs[1:]:
+        for a, b in zip(runs[0], r):
+            assert torch.equal(a, b)
+    f64 = lambda x: x.float().cpu().numpy().astype(np.float64)
+    check_against_oracle(w, tens, (f64(o), f64(lse)) + tuple(f64(x) for x in runs[0]))
+
+
+def test_deterministic_backward_full_size_config1():
+    """The benchmark's configuration: bit-identical dQ over two runs at full size."""
+    from paper_2602_24082_b200 import binding as B
+    w = W.config1()
+    q, k, v, do = (x.cuda() for x in w.tensors())
+    plan = B.plan_for(w, desc_on_device=True)
+    o, lse = B.pp_attn_fwd(plan, q, k, v, w.softmax_scale)
+    a = [x.clone() for x in B.pp_attn_bwd(plan, q, k, v, o, lse, do, w.softmax_scale, deterministic=True)]
+    b = B.pp_attn_bwd(plan, q, k, v, o, lse, do, w.softmax_scale, deterministic=True)
+    c = B.pp_attn_bwd(plan, q, k, v, o, lse, do, w.softmax_scale)
+    torch.cuda.synchronize()
+    assert plan.status() == (0, 0)
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+    d = (a[0].float() - c[0].float()).norm() / c[0].float().norm()
+    assert float(d) < 1e-3
+
+
 def test_backward_clears_its_accumulator_when_the_forward_did_not():
     """One forward that cleared the accumulator, then TWO backward calls: the first skips its
     clearing pass, the second must clear for itself (the accumulator now holds the first

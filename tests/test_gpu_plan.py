@@ -69,7 +69,9 @@ def test_plan_matches_dense_mask(w, desc_on_device):
         groups[g] = (min(lo, s0), max(hi, s0 + l0))
     assert len(btiles) == sum((hi - lo + 127) // 128 for lo, hi in groups.values())
     bcov = np.zeros(T, dtype=int)
-    for (start, ln, vis_end, full_end, gstart, gend, work, _pad) in btiles.tolist():
+    prompt_len = {s0: l0 for (s0, l0, _r, _g, k) in segs if k == 0}   # by group start
+    for (start, ln, vis_end, full_end, gstart, gend, work, npc) in btiles.tolist():
+        assert npc == (prompt_len[gstart] + 127) // 128
         assert 1 <= ln <= 128 and (start - gstart) % 128 == 0 and start + ln <= gend
         assert ln == 128 or start + ln == gend
         assert (gstart, gend) in groups.values()
