@@ -408,6 +408,23 @@ def run_ours(args):
             "tflops": bflops / (statistics.median(dms) * 1e-3) / 1e12,
             "slowdown": statistics.median(dms) / statistics.median(nms)}
 
+        # ---- next row: the row builder (batch sorting + packing into rows) on a synthetic
+        # batch of 4096 preference groups of up to 16K tokens, rows of 16384 tokens
+        import numpy as np
+        rng = np.random.default_rng(17)
+        gP = rng.integers(64, 8000, size=4096).astype(np.int32)
+        goff = (np.arange(4097) * 2).astype(np.int32)
+        grl = rng.integers(16, 4000, size=8192).astype(np.int32)
+        dP, doff, drl = (torch.from_numpy(a).to(dev) for a in (gP, goff, grl))
+        for _ in range(3):
+            rb = B.pp_build_rows(dP, doff, drl, 16384)
+        bms, _ = timed(lambda: (B.pp_build_rows(dP, doff, drl, 16384), 0)[1], 10)
+        extra["row_builder"] = {"ms": statistics.median(bms), "groups": 4096,
+                                "rows": int(rb["row_group_off"].numel()) - 1, "row_capacity": 16384,
+                                "tokens": int(rb["row_tokens"].sum().item()),
+                                "note": "integer work in three small kernels; the time includes the "
+                                        "binding's allocations and its status read-back"}
+
     # ---- the CPU oracle beside it (rank 0, N = 1 only), on a bounded sample
     cpu = None
     if world == 1 and not args.no_cpu_baseline:

@@ -251,6 +251,33 @@ int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_
 int pp_profile_enable(int on);
 int pp_profile_read(float* fwd_kernel_ms, float* bwd_main_kernel_ms);
 
+/*
+ * Row builder: the step before the attention path (Sec. 2.3, applied together with preference
+ * packing in Sec. 4.3).  Groups [prompt | responses] are ordered by total length, longest first
+ * and ties in their original order ("batch sorting"), and consecutive groups of that order
+ * are concatenated into rows of at most row_capacity tokens (packing "up to a maximum sequence
+ * length": next fit).  All pointers are DEVICE pointers; everything runs on `stream`.
+ *   in : grp_prompt_len [G], grp_resp_off [G + 1], resp_len [N]        (int32, as in pp_problem)
+ *   out: order [G]            original index of the group at each position of the new order
+ *        row_group_off [G + 1], num_rows [1]   positions [off[r], off[r + 1]) form row r
+ *        row_tokens [G], row_cost [G]          (int64) tokens and visible query-key pairs per
+ *                                              row (Sec. 3.2.1's attention cost)
+ *        out_prompt_len [G], out_resp_off [G + 1], out_resp_len [N]   descriptors in row order:
+ *                                              with row_group_off they are a pp_problem
+ *        status [2]            0 = fine; 1 = malformed group, 2 = a group alone exceeds the
+ *                              capacity (then num_rows = 0); status[1] = the group
+ * d_workspace: pp_build_rows_workspace_bytes(G) bytes, 256-byte aligned.  G <= 65536.
+ * Errors: PP_ERR_INVALID_ARG, PP_ERR_UNSUPPORTED (G too large), PP_ERR_WORKSPACE_TOO_SMALL,
+ * PP_ERR_ALIGNMENT, PP_ERR_CUDA; the device status is for the caller to read.
+ */
+int pp_build_rows_workspace_bytes(int32_t num_groups, size_t* bytes);
+int pp_build_rows(int32_t num_groups, int32_t num_responses, const int32_t* grp_prompt_len,
+                  const int32_t* grp_resp_off, const int32_t* resp_len, int32_t row_capacity,
+                  void* d_workspace, size_t workspace_bytes, int32_t* order,
+                  int32_t* row_group_off, int32_t* num_rows, int64_t* row_tokens,
+                  int64_t* row_cost, int32_t* out_prompt_len, int32_t* out_resp_off,
+                  int32_t* out_resp_len, int32_t* status, pp_stream_t stream);
+
 const char* pp_error_string(int code);
 
 #ifdef __cplusplus

@@ -26,7 +26,8 @@ EXPORTS = ["pp_plan_workspace_bytes", "pp_build_plan", "pp_plan_status", "pp_des
            "pp_attn_step_host", "pp_profile_enable", "pp_profile_read",
            "pp_attn_bwd_noalloc", "pp_attn_bwd_noalloc_max_bytes", "pp_plan_read_bwd_units",
            "pp_plan_read_bwd_tiles", "pp_attn_bwd_deterministic",
-           "pp_position_ids", "pp_rope_qk", "pp_preference_loss"]
+           "pp_position_ids", "pp_rope_qk", "pp_preference_loss",
+           "pp_build_rows_workspace_bytes", "pp_build_rows"]
 
 
 class PPError(RuntimeError):
@@ -73,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.pp_attn_fwd.argtypes = [vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, sz, vp]
         L.pp_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, sz, vp]
         L.pp_attn_bwd_deterministic.argtypes = L.pp_attn_bwd.argtypes
+        L.pp_build_rows_workspace_bytes.argtypes = [ctypes.c_int32, vp]
+        L.pp_build_rows.argtypes = [ctypes.c_int32, ctypes.c_int32, vp, vp, vp, ctypes.c_int32, vp, sz] + [vp] * 10
         L.pp_step_host_arena_bytes.argtypes = [vp, vp]
         L.pp_attn_step_host.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp, sz, vp]
         L.pp_attn_bwd_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
@@ -400,3 +403,34 @@ def plan_for(workload, device: str = "cuda:0", desc_on_device: bool = False) -> 
     """Convenience: plan of a :class:`workloads.Workload`."""
     return pp_build_plan(workload.descriptors(), workload.num_q_heads, workload.num_kv_heads,
                          workload.head_dim, workload.total_tokens, device, desc_on_device)
+
+
+def pp_build_rows(grp_prompt_len: torch.Tensor, grp_resp_off: torch.Tensor, resp_len: torch.Tensor,
+                  row_capacity: int):
+    """Row builder (batch sorting + packing into rows of at most ``row_capacity`` tokens) on
+    int32 DEVICE tensors.  Returns a dict of device tensors: order, row_group_off (trimmed to
+    rows + 1), row_tokens, row_cost (trimmed to rows), grp_prompt_len, grp_resp_off, resp_len in
+    row order, and ``status`` (code, detail) as Python ints (reading it synchronises)."""
+    dev = grp_prompt_len.device
+    G, N = int(grp_prompt_len.numel()), int(resp_len.numel())
+    for t, n, name in ((grp_prompt_len, G, "grp_prompt_len"), (grp_resp_off, G + 1, "grp_resp_off"),
+                       (resp_len, N, "resp_len")):
+        _chk(t, (n,), torch.int32, name)
+    nbytes = ctypes.c_size_t(0)
+    _check(lib().pp_build_rows_workspace_bytes(G, ctypes.byref(nbytes)), "pp_build_rows_workspace_bytes")
+    ws = torch.empty(nbytes.value, dtype=torch.uint8, device=dev)
+    i32 = lambda n: torch.empty(n, dtype=torch.int32, device=dev)
+    i64 = lambda n: torch.empty(n, dtype=torch.int64, device=dev)
+    order, rgo, nrows, status = i32(G), i32(G + 1), i32(1), i32(2)
+    rtok, rcost = i64(G), i64(G)
+    oP, ooff, orl = i32(G), i32(G + 1), i32(N)
+    with torch.cuda.device(dev):
+        _check(lib().pp_build_rows(G, N, grp_prompt_len.data_ptr(), grp_resp_off.data_ptr(),
+                                   resp_len.data_ptr(), int(row_capacity), ws.data_ptr(), ws.numel(),
+                                   order.data_ptr(), rgo.data_ptr(), nrows.data_ptr(), rtok.data_ptr(),
+                                   rcost.data_ptr(), oP.data_ptr(), ooff.data_ptr(), orl.data_ptr(),
+                                   status.data_ptr(), _stream()), "pp_build_rows")
+    st = status.tolist()
+    r = int(nrows.item())
+    return {"order": order, "row_group_off": rgo[:r + 1], "row_tokens": rtok[:r], "row_cost": rcost[:r],
+            "grp_prompt_len": oP, "grp_resp_off": ooff, "resp_len": orl, "status": (st[0], st[1])}

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpp_attn.so")
-SOURCES = ["pp_api.cu", "pp_plan.cu", "pp_fwd.cu", "pp_bwd.cu", "pp_rope.cu", "pp_loss.cu"]
+SOURCES = ["pp_api.cu", "pp_plan.cu", "pp_fwd.cu", "pp_bwd.cu", "pp_rope.cu", "pp_loss.cu", "pp_rows.cu"]
 HEADERS = ["pp_internal.h", "pp_dev.cuh", "pp_ptx.cuh", os.path.join("..", "..", "include", "pp_attn.h")]
 
 

@@ -385,6 +385,34 @@ int pp_profile_read(float* fwd_kernel_ms, float* bwd_main_kernel_ms) {
   return pp::profile_read(fwd_kernel_ms, bwd_main_kernel_ms) ? PP_OK : PP_ERR_CUDA;
 }
 
+int pp_build_rows_workspace_bytes(int32_t num_groups, size_t* bytes) {
+  if (num_groups < 1 || !bytes) return PP_ERR_INVALID_ARG;
+  *bytes = pp::rows_workspace_bytes(num_groups);
+  return PP_OK;
+}
+
+int pp_build_rows(int32_t num_groups, int32_t num_responses, const int32_t* grp_prompt_len,
+                  const int32_t* grp_resp_off, const int32_t* resp_len, int32_t row_capacity,
+                  void* d_workspace, size_t workspace_bytes, int32_t* order,
+                  int32_t* row_group_off, int32_t* num_rows, int64_t* row_tokens,
+                  int64_t* row_cost, int32_t* out_prompt_len, int32_t* out_resp_off,
+                  int32_t* out_resp_len, int32_t* status, pp_stream_t stream) {
+  g_last_launches = 0;
+  if (num_groups < 1 || num_responses < num_groups || row_capacity < 1 || !grp_prompt_len ||
+      !grp_resp_off || !resp_len || !d_workspace || !order || !row_group_off || !num_rows ||
+      !row_tokens || !row_cost || !out_prompt_len || !out_resp_off || !out_resp_len || !status)
+    return PP_ERR_INVALID_ARG;
+  if (num_groups > 65536) return PP_ERR_UNSUPPORTED;
+  if (workspace_bytes < pp::rows_workspace_bytes(num_groups)) return PP_ERR_WORKSPACE_TOO_SMALL;
+  if (reinterpret_cast<uintptr_t>(d_workspace) & 255) return PP_ERR_ALIGNMENT;
+  cudaError_t e = pp::launch_build_rows(
+      num_groups, num_responses, grp_prompt_len, grp_resp_off, resp_len, row_capacity, d_workspace,
+      order, row_group_off, num_rows, reinterpret_cast<long long*>(row_tokens),
+      reinterpret_cast<long long*>(row_cost), out_prompt_len, out_resp_off, out_resp_len, status,
+      reinterpret_cast<cudaStream_t>(stream), &g_last_launches);
+  return e == cudaSuccess ? PP_OK : PP_ERR_CUDA;
+}
+
 const char* pp_error_string(int code) {
   switch (code) {
     case PP_OK: return "ok";

@@ -181,6 +181,15 @@ cudaError_t launch_bwd(const pp_plan* plan, const void* q, const void* k, const 
                        void* dk, void* dv, void* scratch, bool dq_cleared, bool deterministic,
                        cudaStream_t stream, int* launches);
 
+// Row builder (csrc/pp_rows.cu).
+size_t rows_workspace_bytes(int num_groups);
+cudaError_t launch_build_rows(int G, int N, const int32_t* prompt_len, const int32_t* resp_off,
+                              const int32_t* resp_len, int capacity, void* ws, int32_t* order,
+                              int32_t* row_group_off, int32_t* num_rows, long long* row_tokens,
+                              long long* row_cost, int32_t* out_prompt_len, int32_t* out_resp_off,
+                              int32_t* out_resp_len, int32_t* status, cudaStream_t stream,
+                              int* launches);
+
 // Size of the scratch array built into the library image for pp_attn_bwd_noalloc.
 constexpr size_t kStaticScratchBytes = size_t(32) << 20;
 cudaError_t launch_bwd_static(const pp_plan* plan, const void* q, const void* k, const void* v,
