@@ -21,7 +21,10 @@ struct RowsPtrs {
   long long* tok;    // [G] tokens per group
   long long* cost;   // [G] visible pairs per group
   long long* pre;    // [G] inclusive prefix sums of the sorted groups' tokens
-  int32_t* nresp;    // [G + 1] scan space for the reordered response offsets
+  int32_t* nxt;      // [G] end of the row that would start at each sorted position
+  int32_t* jump_a;   // [G] pointer-doubling buffers
+  int32_t* jump_b;   // [G]
+  int32_t* mark;     // [G] 1 = a row starts here
   int32_t* order;
   int32_t* row_group_off;
   int32_t* num_rows;
@@ -134,25 +137,63 @@ __global__ void __launch_bounds__(1024) rows_pack_kernel(RowsPtrs p) {
     }
     __syncthreads();
   }
-  if (tid == 0) {
-    p.out_resp_off[p.G] = s_carry_b;
-    // next fit: a row takes sorted groups [s, e) with e the largest index whose tokens still fit
-    int rows = 0, s = 0;
-    p.row_group_off[0] = 0;
-    while (s < p.G) {
-      const long long base = s ? p.pre[s - 1] : 0;
-      int lo = s + 1, hi = p.G;  // the row holds at least group s (every group fits alone)
-      while (lo < hi) {           // largest e in [s + 1, G] with pre[e - 1] - base <= capacity
-        const int mid = (lo + hi + 1) >> 1;
-        if (p.pre[mid - 1] - base <= p.capacity) lo = mid; else hi = mid - 1;
-      }
-      p.row_tokens[rows] = p.pre[lo - 1] - base;
-      ++rows;
-      p.row_group_off[rows] = lo;
-      s = lo;
+  if (tid == 0) p.out_resp_off[p.G] = s_carry_b;
+  __syncthreads();
+  // Next fit in parallel.  nxt[s] = where the row that starts at sorted position s ends: the
+  // largest e whose tokens still fit (every group fits alone, so e > s).  The row starts are
+  // the positions reachable from 0 through nxt; they are marked by pointer doubling (after
+  // round r every start within 2^r hops is marked), then numbered by a prefix count.
+  for (int s = tid; s < p.G; s += nthr) {
+    const long long base = s ? p.pre[s - 1] : 0;
+    int lo = s + 1, hi = p.G;
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (p.pre[mid - 1] - base <= p.capacity) lo = mid; else hi = mid - 1;
     }
-    *p.num_rows = rows;
-    s_rows = rows;
+    p.nxt[s] = lo;
+    p.jump_a[s] = lo;
+    p.mark[s] = (s == 0);
+  }
+  int32_t* ja = p.jump_a;
+  int32_t* jb = p.jump_b;
+  for (int hop = 1; hop < p.G; hop <<= 1) {
+    __syncthreads();
+    for (int s = tid; s < p.G; s += nthr)
+      if (p.mark[s] && ja[s] < p.G) p.mark[ja[s]] = 1;
+    for (int s = tid; s < p.G; s += nthr) jb[s] = ja[s] < p.G ? ja[ja[s]] : p.G;
+    __syncthreads();
+    int32_t* t = ja;
+    ja = jb;
+    jb = t;
+  }
+  __syncthreads();
+  // number the marked positions (exclusive scan of the marks) and emit the rows
+  if (tid == 0) s_carry_b = 0;
+  __syncthreads();
+  for (int base = 0; base < p.G; base += nthr) {
+    const int i = base + tid;
+    const int32_t m = i < p.G ? p.mark[i] : 0;
+    s_b[tid] = m;
+    __syncthreads();
+    for (int d = 1; d < nthr; d <<= 1) {
+      const int32_t xb = tid >= d ? s_b[tid - d] : 0;
+      __syncthreads();
+      s_b[tid] += xb;
+      __syncthreads();
+    }
+    if (m) {
+      const int r = s_carry_b + s_b[tid] - 1;
+      p.row_group_off[r] = i;
+      p.row_tokens[r] = p.pre[p.nxt[i] - 1] - (i ? p.pre[i - 1] : 0);
+    }
+    __syncthreads();
+    if (tid == nthr - 1) s_carry_b += s_b[tid];
+    __syncthreads();
+  }
+  if (tid == 0) {
+    p.row_group_off[s_carry_b] = p.G;
+    *p.num_rows = s_carry_b;
+    s_rows = s_carry_b;
   }
   __syncthreads();
   for (int r = tid; r < s_rows; r += nthr) {
@@ -170,7 +211,7 @@ __global__ void __launch_bounds__(1024) rows_pack_kernel(RowsPtrs p) {
 }  // namespace
 
 size_t rows_workspace_bytes(int G) {
-  return align_up(size_t(8) * G, 256) * 3 + align_up(size_t(4) * (G + 1), 256);
+  return align_up(size_t(8) * G, 256) * 3 + align_up(size_t(4) * G, 256) * 4;
 }
 
 cudaError_t launch_build_rows(int G, int N, const int32_t* prompt_len, const int32_t* resp_off,
@@ -191,7 +232,11 @@ cudaError_t launch_build_rows(int G, int N, const int32_t* prompt_len, const int
   p.tok = reinterpret_cast<long long*>(w);
   p.cost = reinterpret_cast<long long*>(w + a8);
   p.pre = reinterpret_cast<long long*>(w + 2 * a8);
-  p.nresp = reinterpret_cast<int32_t*>(w + 3 * a8);
+  const size_t a4 = align_up(size_t(4) * G, 256);
+  p.nxt = reinterpret_cast<int32_t*>(w + 3 * a8);
+  p.jump_a = reinterpret_cast<int32_t*>(w + 3 * a8 + a4);
+  p.jump_b = reinterpret_cast<int32_t*>(w + 3 * a8 + 2 * a4);
+  p.mark = reinterpret_cast<int32_t*>(w + 3 * a8 + 3 * a4);
   p.order = order;
   p.row_group_off = row_group_off;
   p.num_rows = num_rows;
