@@ -229,8 +229,12 @@ int pp_last_launch_count(void);
 /*
  * One whole pass of the hot path on HOST buffers: copies Q, K, V, dO to the device, builds
  * the plan from the host descriptors, runs forward and backward, and copies O, LSE, dQ, dK,
- * dV back -- all enqueued on `stream`; the caller synchronises the stream before reading the
- * outputs.  Host buffers should be page-locked for the copies to be asynchronous.  d_arena
+ * dV back; the caller synchronises `stream` before reading the outputs.  The kernels and
+ * most copies are enqueued on `stream`; the upload of dO and the download of O and LSE run on
+ * two side streams of the library (created once per device) so that copies in opposite
+ * directions overlap each other and the kernels, and `stream` is made to wait for them: once
+ * `stream` has completed, everything has.  Host buffers should be page-locked for the copies
+ * to be asynchronous.  d_arena
  * is caller-owned device memory of at least pp_step_host_arena_bytes (256-byte aligned); it
  * holds the device copies, the plan workspace and the backward scratch.  `problem` must have
  * desc_on_device == 0.  Same layouts and errors as the calls above.

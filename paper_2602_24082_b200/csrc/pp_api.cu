@@ -3,6 +3,8 @@
 #include <new>
 #include <string.h>
 
+#include <mutex>
+
 #include "pp_internal.h"
 
 namespace {
@@ -330,6 +332,36 @@ int pp_step_host_arena_bytes(const pp_problem* problem, size_t* arena_bytes) {
   return PP_OK;
 }
 
+namespace {
+// Side streams and events of pp_attn_step_host, created once per device on first use.
+struct StepStreams {
+  cudaStream_t up = nullptr, down = nullptr;
+  cudaEvent_t e_qkv = nullptr, e_do = nullptr, e_fwd = nullptr, e_out = nullptr;
+};
+StepStreams* step_streams() {
+  constexpr int kMaxDevices = 64;
+  static std::mutex mu;
+  static StepStreams per_device[kMaxDevices];
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  StepStreams& st = per_device[dev];
+  if (!st.up) {
+    bool ok = cudaStreamCreateWithFlags(&st.up, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&st.down, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&st.e_qkv, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&st.e_do, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&st.e_fwd, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&st.e_out, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+      st = StepStreams();
+      return nullptr;
+    }
+  }
+  return &st;
+}
+}  // namespace
+
 int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_k, const void* h_v,
                       const void* h_do, float softmax_scale, void* h_o, float* h_lse, void* h_dq,
                       void* h_dk, void* h_dv, void* d_arena, size_t arena_bytes,
@@ -348,10 +380,18 @@ int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_
   const size_t T = problem->total_tokens, D = problem->head_dim;
   const size_t qb = T * problem->num_q_heads * D * 2, kb = T * problem->num_kv_heads * D * 2;
   const size_t lb = T * problem->num_q_heads * 4;
+  // Copies in opposite directions overlap (and overlap the kernels): dO goes up on a side
+  // stream while the forward runs and O / LSE come down, O and LSE come down on another side
+  // stream while the backward runs.  The caller's stream ends up waiting for both.
+  StepStreams* ss = step_streams();
+  if (!ss) return PP_ERR_CUDA;
   bool ok = cudaMemcpyAsync(base + a.q, h_q, qb, cudaMemcpyHostToDevice, s) == cudaSuccess &&
             cudaMemcpyAsync(base + a.k, h_k, kb, cudaMemcpyHostToDevice, s) == cudaSuccess &&
             cudaMemcpyAsync(base + a.v, h_v, kb, cudaMemcpyHostToDevice, s) == cudaSuccess &&
-            cudaMemcpyAsync(base + a.d_o, h_do, qb, cudaMemcpyHostToDevice, s) == cudaSuccess;
+            cudaEventRecord(ss->e_qkv, s) == cudaSuccess &&
+            cudaStreamWaitEvent(ss->up, ss->e_qkv, 0) == cudaSuccess &&
+            cudaMemcpyAsync(base + a.d_o, h_do, qb, cudaMemcpyHostToDevice, ss->up) == cudaSuccess &&
+            cudaEventRecord(ss->e_do, ss->up) == cudaSuccess;
   if (!ok) return PP_ERR_CUDA;
   pp_plan* plan = nullptr;
   rc = pp_build_plan(problem, base + a.plan, a.scratch - a.plan, stream, &plan);
@@ -362,6 +402,15 @@ int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_
                    stream);
   launches += g_last_launches;
   if (rc == PP_OK) {
+    ok = cudaEventRecord(ss->e_fwd, s) == cudaSuccess &&
+         cudaStreamWaitEvent(ss->down, ss->e_fwd, 0) == cudaSuccess &&
+         cudaMemcpyAsync(h_o, base + a.o, qb, cudaMemcpyDeviceToHost, ss->down) == cudaSuccess &&
+         cudaMemcpyAsync(h_lse, base + a.lse, lb, cudaMemcpyDeviceToHost, ss->down) == cudaSuccess &&
+         cudaEventRecord(ss->e_out, ss->down) == cudaSuccess &&
+         cudaStreamWaitEvent(s, ss->e_do, 0) == cudaSuccess;
+    if (!ok) rc = PP_ERR_CUDA;
+  }
+  if (rc == PP_OK) {
     rc = pp_attn_bwd(plan, base + a.q, base + a.k, base + a.v, base + a.o,
                      reinterpret_cast<float*>(base + a.lse), base + a.d_o, softmax_scale,
                      base + a.dq, base + a.dk, base + a.dv, base + a.scratch, a.total - a.scratch,
@@ -371,11 +420,10 @@ int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_
   pp_destroy_plan(plan);
   g_last_launches = launches;
   if (rc) return rc;
-  ok = cudaMemcpyAsync(h_o, base + a.o, qb, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
-       cudaMemcpyAsync(h_lse, base + a.lse, lb, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
-       cudaMemcpyAsync(h_dq, base + a.dq, qb, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
+  ok = cudaMemcpyAsync(h_dq, base + a.dq, qb, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
        cudaMemcpyAsync(h_dk, base + a.dk, kb, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
-       cudaMemcpyAsync(h_dv, base + a.dv, kb, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+       cudaMemcpyAsync(h_dv, base + a.dv, kb, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
+       cudaStreamWaitEvent(s, ss->e_out, 0) == cudaSuccess;
   return ok ? PP_OK : PP_ERR_CUDA;
 }
 
