@@ -216,7 +216,7 @@ __device__ __forceinline__ QTile q_tile_at(const BwdParams& prm, const BwdUnit& 
   return q;
 }
 
-template <int D>
+template <int D, bool kDet>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
            const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
@@ -616,12 +616,12 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       // waited for is always running or done and the waits cannot lock up.
       const int k_rel = (un.tile.start - un.tile.grp_start) / kTile;
       int prev_vis_end = 0;
-      if (prm.dq_sem && leader && k_rel > 0) prev_vis_end = prm.tiles[un.tidx - 1].vis_end;
+      if (kDet && leader && k_rel > 0) prev_vis_end = prm.tiles[un.tidx - 1].vis_end;
       for (int it = 0; it < un.n_it; ++it, q_advance(qi, prm.Hq / prm.Hkv)) {
         const QTile qt = q_tile_at(prm, un, qi);
         const uint32_t g = gc + it;
         int32_t* sem = nullptr;
-        if (prm.dq_sem && leader) sem = prm.dq_sem + size_t(un.tidx + qi.qt) * prm.Hq + qt.h;
+        if (kDet && leader) sem = prm.dq_sem + size_t(un.tidx + qi.qt) * prm.Hq + qt.h;
         wait_bar(bar(kDqFull), g & 1, abort_flag, prm.header, 80);
         tc_fence_after();
         // Two halves of D/2 columns.  The second half is read out of tensor memory (and the
@@ -661,7 +661,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             fence_proxy_async_smem();
             named_barrier_sync(1, 128);
             if (leader) {
-              if (sem && half == 0 && c == 0) {  // wait for this unit's turn (bounded)
+              if (kDet && sem && half == 0 && c == 0) {  // wait for this unit's turn (bounded)
                 const int expect =
                     k_rel == 0 ? 0 : (prev_vis_end > qt.start ? k_rel : un.tile.npc);
                 bool ok = false;
@@ -686,7 +686,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             }
           }
         }
-        if (sem) {  // all four boxes of the tile added and visible: pass the turn on
+        if (kDet && sem) {  // all four boxes of the tile added and visible: pass the turn on
           bulk_wait_group<0>();
           __threadfence();
           const int mine = k_rel + 1;
@@ -740,10 +740,14 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
                          const BwdParams& prm, bool dq_cleared, cudaStream_t stream,
                          int* launches) {
   static bool configured = false;
-  auto kern = bwd_kernel<D>;
+  auto kern = prm.dq_sem ? bwd_kernel<D, true> : bwd_kernel<D, false>;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(bwd_kernel<D, false>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          BwdSmem<D>::kTotal);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(bwd_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               BwdSmem<D>::kTotal);
     if (e != cudaSuccess) return e;
     configured = true;
   }
