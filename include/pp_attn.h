@@ -229,15 +229,19 @@ int pp_last_launch_count(void);
 /*
  * One whole pass of the hot path on HOST buffers: copies Q, K, V, dO to the device, builds
  * the plan from the host descriptors, runs forward and backward, and copies O, LSE, dQ, dK,
- * dV back; the caller synchronises `stream` before reading the outputs.  The kernels and
- * most copies are enqueued on `stream`; the upload of dO and the download of O and LSE run on
- * two side streams of the library (created once per device) so that copies in opposite
- * directions overlap each other and the kernels, and `stream` is made to wait for them: once
- * `stream` has completed, everything has.  Host buffers should be page-locked for the copies
- * to be asynchronous.  d_arena
- * is caller-owned device memory of at least pp_step_host_arena_bytes (256-byte aligned); it
- * holds the device copies, the plan workspace and the backward scratch.  `problem` must have
- * desc_on_device == 0.  Same layouts and errors as the calls above.
+ * dV back; the caller synchronises `stream` before reading the outputs.  Groups never interact
+ * (paper section 3), so the pass is cut into up to eight runs of whole groups with about equal
+ * token counts (fewer when a run would hold under a quarter MiB of input), each with its own plan, and pipelined: the kernels run on `stream`, all
+ * uploads on one side stream of the library and all downloads on another (both created once
+ * per device), so that the inputs of the next run go up and the results of the previous run
+ * come down, in opposite directions, while the kernels of the current run execute.  `stream`
+ * is made to wait for both side streams: once `stream` has completed, everything has.  The
+ * results are those of one pp_attn_fwd + pp_attn_bwd over the whole problem (dK, dV, O and
+ * LSE bit for bit).  Host buffers should be page-locked for the copies to be asynchronous.
+ * d_arena is caller-owned device memory of at least pp_step_host_arena_bytes (256-byte
+ * aligned); it holds the device copies, the plan workspaces and the backward scratch.
+ * `problem` must have desc_on_device == 0; its descriptors are validated on the host first.
+ * Same layouts and errors as the calls above.
  */
 int pp_step_host_arena_bytes(const pp_problem* problem, size_t* arena_bytes);
 int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_k, const void* h_v,

@@ -3,7 +3,9 @@
 #include <new>
 #include <string.h>
 
+#include <algorithm>
 #include <mutex>
+#include <vector>
 
 #include "pp_internal.h"
 
@@ -336,7 +338,9 @@ namespace {
 // Side streams and events of pp_attn_step_host, created once per device on first use.
 struct StepStreams {
   cudaStream_t up = nullptr, down = nullptr;
-  cudaEvent_t e_qkv = nullptr, e_do = nullptr, e_fwd = nullptr, e_out = nullptr;
+  cudaEvent_t e_start = nullptr, e_end = nullptr;
+  cudaEvent_t e_qkv[pp::kStepChunks] = {}, e_do[pp::kStepChunks] = {}, e_fwd[pp::kStepChunks] = {},
+              e_bwd[pp::kStepChunks] = {};
 };
 StepStreams* step_streams() {
   constexpr int kMaxDevices = 64;
@@ -347,18 +351,88 @@ StepStreams* step_streams() {
   std::lock_guard<std::mutex> lock(mu);
   StepStreams& st = per_device[dev];
   if (!st.up) {
+    auto ev = [](cudaEvent_t* e) {
+      return cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
+    };
     bool ok = cudaStreamCreateWithFlags(&st.up, cudaStreamNonBlocking) == cudaSuccess &&
               cudaStreamCreateWithFlags(&st.down, cudaStreamNonBlocking) == cudaSuccess &&
-              cudaEventCreateWithFlags(&st.e_qkv, cudaEventDisableTiming) == cudaSuccess &&
-              cudaEventCreateWithFlags(&st.e_do, cudaEventDisableTiming) == cudaSuccess &&
-              cudaEventCreateWithFlags(&st.e_fwd, cudaEventDisableTiming) == cudaSuccess &&
-              cudaEventCreateWithFlags(&st.e_out, cudaEventDisableTiming) == cudaSuccess;
+              ev(&st.e_start) && ev(&st.e_end);
+    for (int c = 0; ok && c < pp::kStepChunks; ++c)
+      ok = ev(&st.e_qkv[c]) && ev(&st.e_do[c]) && ev(&st.e_fwd[c]) && ev(&st.e_bwd[c]);
     if (!ok) {
       st = StepStreams();
       return nullptr;
     }
   }
   return &st;
+}
+
+// One run of whole rows of a step: its descriptors (rebased to start at zero), its token range
+// and where its private blocks sit in the arena.
+struct StepChunk {
+  std::vector<int32_t> row_group_off, grp_resp_off;
+  pp_problem prob{};
+  size_t t0 = 0, plan_off = 0, plan_bytes = 0, scratch_off = 0, scratch_bytes = 0, lse_off = 0;
+};
+
+// Cuts `p` (host descriptors, already validated) into at most `want` runs of whole groups with
+// about equal token counts.  Groups never interact, so a row that is cut becomes two rows.
+std::vector<StepChunk> cut_step(const pp_problem& p, int want) {
+  std::vector<size_t> grp_end(p.num_groups);
+  size_t t = 0;
+  for (int g = 0; g < p.num_groups; ++g) {
+    t += p.grp_prompt_len[g];
+    for (int i = p.grp_resp_off[g]; i < p.grp_resp_off[g + 1]; ++i) t += p.resp_len[i];
+    grp_end[g] = t;
+  }
+  const int n = std::max(1, std::min(want, p.num_groups));
+  std::vector<StepChunk> out;
+  int g0 = 0, r = 0;
+  for (int c = 0; c < n && g0 < p.num_groups; ++c) {
+    int g1 = g0 + 1;
+    const size_t target = t * size_t(c + 1) / size_t(n);
+    // leave at least one group for every later run
+    while (g1 < p.num_groups - (n - 1 - c) && grp_end[g1 - 1] < target) ++g1;
+    if (c == n - 1) g1 = p.num_groups;
+    StepChunk ch;
+    const int i0 = p.grp_resp_off[g0], i1 = p.grp_resp_off[g1];
+    ch.row_group_off.push_back(0);
+    while (p.row_group_off[r + 1] <= g0) ++r;
+    for (int rr = r; rr < p.num_rows && p.row_group_off[rr] < g1; ++rr)
+      ch.row_group_off.push_back(std::min(p.row_group_off[rr + 1], g1) - g0);
+    for (int g = g0; g <= g1; ++g) ch.grp_resp_off.push_back(p.grp_resp_off[g] - i0);
+    ch.t0 = g0 ? grp_end[g0 - 1] : 0;
+    ch.prob = p;
+    ch.prob.num_rows = int32_t(ch.row_group_off.size()) - 1;
+    ch.prob.num_groups = g1 - g0;
+    ch.prob.num_responses = i1 - i0;
+    ch.prob.total_tokens = int32_t(grp_end[g1 - 1] - ch.t0);
+    ch.prob.grp_prompt_len = p.grp_prompt_len + g0;
+    ch.prob.resp_len = p.resp_len + i0;
+    out.push_back(std::move(ch));
+    g0 = g1;
+  }
+  for (StepChunk& ch : out) {   // the vectors no longer move
+    ch.prob.row_group_off = ch.row_group_off.data();
+    ch.prob.grp_resp_off = ch.grp_resp_off.data();
+  }
+  return out;
+}
+
+// Places the chunks' private blocks; false if they do not fit the arena's regions.
+bool place_step(std::vector<StepChunk>& chunks, const pp::StepArena& a, size_t heads_q) {
+  size_t po = a.plan, so = a.scratch, lo = a.lse;
+  for (StepChunk& ch : chunks) {
+    ch.plan_off = po;
+    ch.plan_bytes = pp::plan_layout(ch.prob).total;
+    po += pp::align_up(ch.plan_bytes, 256);
+    ch.scratch_off = so;
+    ch.scratch_bytes = pp::bwd_scratch_layout(ch.prob).total;
+    so += pp::align_up(ch.scratch_bytes, 256);
+    ch.lse_off = lo;
+    lo += pp::align_up(size_t(ch.prob.total_tokens) * heads_q * 4, 256);
+  }
+  return po <= a.scratch && so <= a.total && lo <= a.dq;
 }
 }  // namespace
 
@@ -372,59 +446,107 @@ int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_
   if (problem->desc_on_device) return PP_ERR_INVALID_ARG;
   if (!h_q || !h_k || !h_v || !h_do || !h_o || !h_lse || !h_dq || !h_dk || !h_dv || !d_arena)
     return PP_ERR_INVALID_ARG;
+  if (!problem->row_group_off || !problem->grp_prompt_len || !problem->grp_resp_off ||
+      !problem->resp_len)
+    return PP_ERR_INVALID_ARG;
+  rc = check_host_descriptors(problem);
+  if (rc) return rc;
   if (reinterpret_cast<uintptr_t>(d_arena) & 255) return PP_ERR_ALIGNMENT;
-  pp::StepArena a = pp::step_arena_layout(*problem);
+  const pp::StepArena a = pp::step_arena_layout(*problem);
   if (arena_bytes < a.total) return PP_ERR_WORKSPACE_TOO_SMALL;
+  StepStreams* ss = step_streams();
+  if (!ss) return PP_ERR_CUDA;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   char* base = static_cast<char*>(d_arena);
   const size_t T = problem->total_tokens, D = problem->head_dim;
-  const size_t qb = T * problem->num_q_heads * D * 2, kb = T * problem->num_kv_heads * D * 2;
-  const size_t lb = T * problem->num_q_heads * 4;
-  // Copies in opposite directions overlap (and overlap the kernels): dO goes up on a side
-  // stream while the forward runs and O / LSE come down, O and LSE come down on another side
-  // stream while the backward runs.  The caller's stream ends up waiting for both.
-  StepStreams* ss = step_streams();
-  if (!ss) return PP_ERR_CUDA;
-  bool ok = cudaMemcpyAsync(base + a.q, h_q, qb, cudaMemcpyHostToDevice, s) == cudaSuccess &&
-            cudaMemcpyAsync(base + a.k, h_k, kb, cudaMemcpyHostToDevice, s) == cudaSuccess &&
-            cudaMemcpyAsync(base + a.v, h_v, kb, cudaMemcpyHostToDevice, s) == cudaSuccess &&
-            cudaEventRecord(ss->e_qkv, s) == cudaSuccess &&
-            cudaStreamWaitEvent(ss->up, ss->e_qkv, 0) == cudaSuccess &&
-            cudaMemcpyAsync(base + a.d_o, h_do, qb, cudaMemcpyHostToDevice, ss->up) == cudaSuccess &&
-            cudaEventRecord(ss->e_do, ss->up) == cudaSuccess;
-  if (!ok) return PP_ERR_CUDA;
-  pp_plan* plan = nullptr;
-  rc = pp_build_plan(problem, base + a.plan, a.scratch - a.plan, stream, &plan);
-  if (rc) return rc;
-  int launches = g_last_launches;
-  rc = pp_attn_fwd(plan, base + a.q, base + a.k, base + a.v, softmax_scale, base + a.o,
-                   reinterpret_cast<float*>(base + a.lse), base + a.scratch, a.total - a.scratch,
-                   stream);
-  launches += g_last_launches;
-  if (rc == PP_OK) {
-    ok = cudaEventRecord(ss->e_fwd, s) == cudaSuccess &&
-         cudaStreamWaitEvent(ss->down, ss->e_fwd, 0) == cudaSuccess &&
-         cudaMemcpyAsync(h_o, base + a.o, qb, cudaMemcpyDeviceToHost, ss->down) == cudaSuccess &&
-         cudaMemcpyAsync(h_lse, base + a.lse, lb, cudaMemcpyDeviceToHost, ss->down) == cudaSuccess &&
-         cudaEventRecord(ss->e_out, ss->down) == cudaSuccess &&
-         cudaStreamWaitEvent(s, ss->e_do, 0) == cudaSuccess;
-    if (!ok) rc = PP_ERR_CUDA;
+  const size_t Hq = problem->num_q_heads, Hkv = problem->num_kv_heads;
+
+  // Groups are independent, so the step runs as a short pipeline over runs of whole groups: the
+  // inputs of run c+1 go up and the results of run c-1 come down (two copy engines, opposite
+  // directions) while the kernels of run c execute.  Inside a run dO still goes up behind
+  // the forward and O / LSE come down behind the backward.
+  // A run below a quarter MiB of input is all launch overhead: fewer runs then.
+  const size_t in_bytes = T * (Hq + Hkv) * D * 4;
+  const int want = int(std::min<size_t>(pp::kStepChunks, std::max<size_t>(1, in_bytes >> 18)));
+  std::vector<StepChunk> chunks = cut_step(*problem, want);
+  if (!place_step(chunks, a, Hq)) {
+    chunks = cut_step(*problem, 1);
+    if (!place_step(chunks, a, Hq)) return PP_ERR_WORKSPACE_TOO_SMALL;
   }
-  if (rc == PP_OK) {
-    rc = pp_attn_bwd(plan, base + a.q, base + a.k, base + a.v, base + a.o,
-                     reinterpret_cast<float*>(base + a.lse), base + a.d_o, softmax_scale,
-                     base + a.dq, base + a.dk, base + a.dv, base + a.scratch, a.total - a.scratch,
-                     stream);
+  auto ok = [](cudaError_t e) { return e == cudaSuccess; };
+  if (!ok(cudaEventRecord(ss->e_start, s)) || !ok(cudaStreamWaitEvent(ss->up, ss->e_start, 0)) ||
+      !ok(cudaStreamWaitEvent(ss->down, ss->e_start, 0)))
+    return PP_ERR_CUDA;
+  int launches = 0;
+  const char* hq = static_cast<const char*>(h_q);
+  const char* hk = static_cast<const char*>(h_k);
+  const char* hv = static_cast<const char*>(h_v);
+  const char* hdo = static_cast<const char*>(h_do);
+  for (size_t c = 0; c < chunks.size(); ++c) {      // all uploads, in order, on the `up` stream
+    const StepChunk& ch = chunks[c];
+    const size_t tc = ch.prob.total_tokens;
+    const size_t qo = ch.t0 * Hq * D * 2, ko = ch.t0 * Hkv * D * 2;
+    const size_t qb = tc * Hq * D * 2, kb = tc * Hkv * D * 2;
+    if (!ok(cudaMemcpyAsync(base + a.q + qo, hq + qo, qb, cudaMemcpyHostToDevice, ss->up)) ||
+        !ok(cudaMemcpyAsync(base + a.k + ko, hk + ko, kb, cudaMemcpyHostToDevice, ss->up)) ||
+        !ok(cudaMemcpyAsync(base + a.v + ko, hv + ko, kb, cudaMemcpyHostToDevice, ss->up)) ||
+        !ok(cudaEventRecord(ss->e_qkv[c], ss->up)) ||
+        !ok(cudaMemcpyAsync(base + a.d_o + qo, hdo + qo, qb, cudaMemcpyHostToDevice, ss->up)) ||
+        !ok(cudaEventRecord(ss->e_do[c], ss->up)))
+      return PP_ERR_CUDA;
+  }
+  for (size_t c = 0; c < chunks.size() && rc == PP_OK; ++c) {
+    const StepChunk& ch = chunks[c];
+    const size_t tc = ch.prob.total_tokens;
+    const size_t qo = ch.t0 * Hq * D * 2, ko = ch.t0 * Hkv * D * 2;
+    const size_t qb = tc * Hq * D * 2, kb = tc * Hkv * D * 2;
+    float* d_lse = reinterpret_cast<float*>(base + ch.lse_off);
+    pp_plan* plan = nullptr;
+    rc = pp_build_plan(&ch.prob, base + ch.plan_off, ch.plan_bytes, stream, &plan);
+    if (rc) break;
     launches += g_last_launches;
+    if (!ok(cudaStreamWaitEvent(s, ss->e_qkv[c], 0))) rc = PP_ERR_CUDA;
+    if (rc == PP_OK) {
+      rc = pp_attn_fwd(plan, base + a.q + qo, base + a.k + ko, base + a.v + ko, softmax_scale,
+                       base + a.o + qo, d_lse, base + ch.scratch_off, ch.scratch_bytes, stream);
+      launches += g_last_launches;
+    }
+    if (rc == PP_OK) {
+      // LSE is [Hq][tokens of the run] on the device and [Hq][T] on the host
+      bool good =
+          ok(cudaEventRecord(ss->e_fwd[c], s)) && ok(cudaStreamWaitEvent(ss->down, ss->e_fwd[c], 0)) &&
+          ok(cudaMemcpyAsync(static_cast<char*>(h_o) + qo, base + a.o + qo, qb,
+                             cudaMemcpyDeviceToHost, ss->down)) &&
+          ok(cudaMemcpy2DAsync(h_lse + ch.t0, T * 4, d_lse, tc * 4, tc * 4, Hq,
+                               cudaMemcpyDeviceToHost, ss->down)) &&
+          ok(cudaStreamWaitEvent(s, ss->e_do[c], 0));
+      if (!good) rc = PP_ERR_CUDA;
+    }
+    if (rc == PP_OK) {
+      rc = pp_attn_bwd(plan, base + a.q + qo, base + a.k + ko, base + a.v + ko, base + a.o + qo,
+                       d_lse, base + a.d_o + qo, softmax_scale, base + a.dq + qo, base + a.dk + ko,
+                       base + a.dv + ko, base + ch.scratch_off, ch.scratch_bytes, stream);
+      launches += g_last_launches;
+    }
+    pp_destroy_plan(plan);
+    if (rc == PP_OK) {
+      bool good =
+          ok(cudaEventRecord(ss->e_bwd[c], s)) && ok(cudaStreamWaitEvent(ss->down, ss->e_bwd[c], 0)) &&
+          ok(cudaMemcpyAsync(static_cast<char*>(h_dq) + qo, base + a.dq + qo, qb,
+                             cudaMemcpyDeviceToHost, ss->down)) &&
+          ok(cudaMemcpyAsync(static_cast<char*>(h_dk) + ko, base + a.dk + ko, kb,
+                             cudaMemcpyDeviceToHost, ss->down)) &&
+          ok(cudaMemcpyAsync(static_cast<char*>(h_dv) + ko, base + a.dv + ko, kb,
+                             cudaMemcpyDeviceToHost, ss->down));
+      if (!good) rc = PP_ERR_CUDA;
+    }
   }
-  pp_destroy_plan(plan);
+  // the caller's stream ends behind everything the side streams were given, also on failure
+  bool joined = ok(cudaEventRecord(ss->e_end, ss->down)) && ok(cudaStreamWaitEvent(s, ss->e_end, 0)) &&
+                ok(cudaEventRecord(ss->e_end, ss->up)) && ok(cudaStreamWaitEvent(s, ss->e_end, 0));
   g_last_launches = launches;
   if (rc) return rc;
-  ok = cudaMemcpyAsync(h_dq, base + a.dq, qb, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
-       cudaMemcpyAsync(h_dk, base + a.dk, kb, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
-       cudaMemcpyAsync(h_dv, base + a.dv, kb, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
-       cudaStreamWaitEvent(s, ss->e_out, 0) == cudaSuccess;
-  return ok ? PP_OK : PP_ERR_CUDA;
+  return joined ? PP_OK : PP_ERR_CUDA;
 }
 
 int pp_profile_enable(int on) { return pp::profile_enable(on != 0) ? PP_OK : PP_ERR_CUDA; }

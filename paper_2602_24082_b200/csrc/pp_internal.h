@@ -143,7 +143,10 @@ inline BwdScratch bwd_scratch_layout(const pp_problem& p) {
   return s;
 }
 
-// Device arena of pp_attn_step_host: inputs, outputs, plan workspace, backward scratch.
+// Device arena of pp_attn_step_host: inputs, outputs, plan workspace, backward scratch.  The
+// step is cut into at most kStepChunks runs of whole groups, each with its own plan, scratch and
+// LSE block inside the shared regions; the regions carry the alignment slack that costs.
+constexpr int kStepChunks = 8;
 struct StepArena {
   size_t q, k, v, d_o, o, lse, dq, dk, dv, plan, scratch, total;
 };
@@ -154,10 +157,10 @@ inline StepArena step_arena_layout(const pp_problem& p) {
   size_t off = 0;
   auto take = [&](size_t n) { size_t o = off; off = align_up(off + n, 256); return o; };
   a.q = take(qb); a.k = take(kb); a.v = take(kb); a.d_o = take(qb);
-  a.o = take(qb); a.lse = take(T * p.num_q_heads * 4);
+  a.o = take(qb); a.lse = take(T * p.num_q_heads * 4 + 256 * kStepChunks);
   a.dq = take(qb); a.dk = take(kb); a.dv = take(kb);
-  a.plan = take(plan_layout(p).total);
-  a.scratch = take(bwd_scratch_layout(p).total);
+  a.plan = take(plan_layout(p).total + size_t(16384) * kStepChunks);
+  a.scratch = take(bwd_scratch_layout(p).total + size_t(4096) * kStepChunks);
   a.total = off;
   return a;
 }

@@ -280,11 +280,23 @@ def test_outputs_outside_tiles_untouched():
         assert (b[:pad] == 7.0).all() and (b[pad + T:] == 7.0).all(), name
 
 
-def test_host_step_matches_the_device_path():
-    """pp_attn_step_host (copies overlapped on side streams) called twice back to back on the
-    same arena: both results equal the device-resident path (forward, dK, dV bit for bit)."""
+HOST_CASES = [
+    W.Workload("host3", [[(300, (140, 77))], [(64, (200, 1))], [(129, (640,))]], 4, 2, 128, seed=31),
+    W.Workload("host1", [[(200, (130, 5)), (3, (1,))]], 2, 1, 64, seed=32),
+    W.Workload("host7", [[(10 + 37 * i, (3 + 50 * (i % 3), 1 + 20 * i)), (64 + i, (9, 130))]
+                         for i in range(7)], 6, 2, 128, seed=33),
+    W.Workload("host-lopsided", [[(1, (1,))], [(900, (300, 300))], [(2, (1, 1))], [(1, (2,))],
+                                 [(5, (5,))], [(400, (1,))]], 2, 2, 128, seed=34),
+]
+
+
+@pytest.mark.parametrize("w", HOST_CASES, ids=lambda w: w.name)
+def test_host_step_matches_the_device_path(w):
+    """pp_attn_step_host (the step cut into runs of whole groups, copies overlapped on side
+    streams) called twice back to back on the same arena: both results equal the
+    device-resident path (forward, dK, dV bit for bit), for fewer groups than runs, more
+    groups than runs (rows cut in the middle) and groups of very different sizes."""
     from paper_2602_24082_b200 import binding as B
-    w = W.Workload("host", [[(300, (140, 77))], [(64, (200, 1))], [(129, (640,))]], 4, 2, 128, seed=31)
     tens = w.tensors()
     ref = _run_gpu(w, tens)
     hs = B.HostStep(w)
