@@ -83,6 +83,11 @@ int pp_plan_workspace_bytes(const pp_problem* problem, size_t* plan_bytes,
  * the backward pass processes (tile, KV head) units group by group (largest group first,
  * longest tile first inside a group) so that concurrently running units share Q / dO in L2.
  * Both kernels draw units dynamically, so the order is a priority list, not an assignment.
+ * Host descriptors (desc_on_device == 0) are validated on the host and staged in the
+ * workspace: up to 7168 entries over the four arrays travel as the argument of a small kernel,
+ * so the call never waits on the host for work already in `stream`; longer ones are copied
+ * with cudaMemcpyAsync, which for pageable host memory does wait for the stream first.  The
+ * host arrays may be changed or freed as soon as the call returns.
  * d_workspace must stay alive and untouched while the plan is used.  The plan is
  * immutable and can be reused by any number of pp_attn_fwd / pp_attn_bwd calls whose
  * tensors have the shapes stated in `problem`.

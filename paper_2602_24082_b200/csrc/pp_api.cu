@@ -1,5 +1,6 @@
 // C ABI of the preference-packed attention library: argument checking, plan handle,
-// workspace bookkeeping.  All device work is enqueued by the launchers in the other files.
+// workspace bookkeeping.  Apart from the kernel that stages host descriptors, all device work
+// is enqueued by the launchers in the other files.
 #include <new>
 #include <string.h>
 
@@ -14,6 +15,30 @@ namespace {
 thread_local int g_last_launches = 0;
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+// Host descriptors handed to the device as a kernel argument (no copy engine, no host-side
+// wait): two sizes so that small batches do not pay for a large argument block.
+constexpr size_t kDescSmall = 960, kDescLarge = 7168;
+template <size_t N>
+struct DescBlock {
+  int32_t v[N];
+};
+template <size_t N>
+__global__ void stage_desc_kernel(const __grid_constant__ DescBlock<N> blk, int n, int32_t* dst) {
+  for (int i = threadIdx.x; i < n; i += blockDim.x) dst[i] = blk.v[i];
+}
+template <size_t N>
+cudaError_t stage_descriptors(const int32_t* const (&src)[4], const size_t (&n)[4], int32_t* dst,
+                              cudaStream_t s) {
+  DescBlock<N> blk;
+  size_t at = 0;
+  for (int i = 0; i < 4; ++i) {
+    memcpy(blk.v + at, src[i], n[i] * sizeof(int32_t));
+    at += n[i];
+  }
+  stage_desc_kernel<N><<<1, 256, 0, s>>>(blk, int(at), dst);
+  return cudaGetLastError();
+}
 
 int check_problem_shape(const pp_problem* p) {
   if (!p) return PP_ERR_INVALID_ARG;
@@ -95,29 +120,41 @@ int pp_build_plan(const pp_problem* problem, void* d_workspace, size_t workspace
   plan->bwd_scratch = pp::bwd_scratch_layout(*problem).total;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
 
+  g_last_launches = 0;
   if (!problem->desc_on_device) {
-    // stage the four arrays in the workspace; the plan kernels read them from there
+    // Stage the four arrays, back to back, in the workspace; the plan kernels read them from
+    // there.  Up to kDescLarge entries travel as the argument of a small kernel, which keeps
+    // the call asynchronous (a cudaMemcpyAsync from pageable host memory would first wait on
+    // the host for everything already in the stream); longer descriptor sets are copied.
     int32_t* d = reinterpret_cast<int32_t*>(plan->ws + lay.desc);
     const int32_t* src[4] = {problem->row_group_off, problem->grp_prompt_len,
                              problem->grp_resp_off, problem->resp_len};
-    size_t n[4] = {size_t(problem->num_rows) + 1, size_t(problem->num_groups),
-                   size_t(problem->num_groups) + 1, size_t(problem->num_responses)};
-    const int32_t* dst[4];
-    for (int i = 0; i < 4; ++i) {
-      cudaError_t e = cudaMemcpyAsync(d, src[i], n[i] * sizeof(int32_t), cudaMemcpyHostToDevice, s);
-      if (e != cudaSuccess) {
-        delete plan;
-        return PP_ERR_CUDA;
+    const size_t n[4] = {size_t(problem->num_rows) + 1, size_t(problem->num_groups),
+                         size_t(problem->num_groups) + 1, size_t(problem->num_responses)};
+    const size_t n_all = n[0] + n[1] + n[2] + n[3];
+    cudaError_t e = cudaSuccess;
+    if (n_all <= kDescSmall) {
+      e = stage_descriptors<kDescSmall>(src, n, d, s);
+      g_last_launches = 1;
+    } else if (n_all <= kDescLarge) {
+      e = stage_descriptors<kDescLarge>(src, n, d, s);
+      g_last_launches = 1;
+    } else {
+      int32_t* at = d;
+      for (int i = 0; i < 4 && e == cudaSuccess; ++i) {
+        e = cudaMemcpyAsync(at, src[i], n[i] * sizeof(int32_t), cudaMemcpyHostToDevice, s);
+        at += n[i];
       }
-      dst[i] = d;
-      d += n[i];
     }
-    plan->prob.row_group_off = dst[0];
-    plan->prob.grp_prompt_len = dst[1];
-    plan->prob.grp_resp_off = dst[2];
-    plan->prob.resp_len = dst[3];
+    if (e != cudaSuccess) {
+      delete plan;
+      return PP_ERR_CUDA;
+    }
+    plan->prob.row_group_off = d;
+    plan->prob.grp_prompt_len = d + n[0];
+    plan->prob.grp_resp_off = d + n[0] + n[1];
+    plan->prob.resp_len = d + n[0] + n[1] + n[2];
   }
-  g_last_launches = 0;
   if (pp::launch_plan(plan, s, &g_last_launches) != cudaSuccess) {
     delete plan;
     return PP_ERR_CUDA;

@@ -178,3 +178,23 @@ def test_device_side_validation_reports_status():
     B.pp_attn_fwd(plan, q, k, v, 0.125, o=o)
     torch.cuda.synchronize()
     assert (o == 3.0).all()
+
+
+@pytest.mark.parametrize("groups", [40, 1100, 2500], ids=["small-block", "large-block", "copied"])
+def test_host_descriptors_reach_the_device_unchanged(groups):
+    """Host descriptors travel as a kernel argument (two block sizes) or, beyond that, by
+    copies: each route gives the plan that device-resident descriptors give."""
+    from paper_2602_24082_b200 import binding as B
+    rows = [[(1 + (i % 7), (1 + (i % 2),)) for i in range(groups)]]
+    w = W.Workload("desc", rows, 2, 1, 64, seed=2)
+    got = B.plan_for(w, desc_on_device=False)
+    want = B.plan_for(w, desc_on_device=True)
+    assert got.status() == (0, 0) and want.status() == (0, 0)
+    nb = len(want.read_bwd_tiles())
+    assert np.array_equal(got.read_bwd_tiles(), want.read_bwd_tiles())
+    for a, b in zip(got.read(), want.read()):   # (tiles, fwd_order, bwd_order, key_end)
+        assert a.shape == b.shape
+    (t0, f0, b0, k0), (t1, f1, b1, k1) = got.read(), want.read()
+    assert np.array_equal(t0, t1) and np.array_equal(f0, f1) and np.array_equal(k0, k1)
+    assert np.array_equal(b0[:nb], b1[:nb])      # entries past the backward tiles are unused
+    assert np.array_equal(got.read_bwd_units(nb), want.read_bwd_units(nb))
