@@ -259,7 +259,8 @@ int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_
  * CUDA events on the caller's stream directly around the forward kernel and around the
  * backward main kernel; pp_profile_read returns the two durations (ms) of the most recent
  * calls once that stream has been synchronised by the caller (PP_ERR_CUDA otherwise).
- * pp_profile_enable(0) releases the events.
+ * pp_profile_enable(0) releases the events.  One set of events per process, created on the
+ * device that is current at pp_profile_enable(1): profile one device at a time.
  */
 int pp_profile_enable(int on);
 int pp_profile_read(float* fwd_kernel_ms, float* bwd_main_kernel_ms);

@@ -380,11 +380,10 @@ struct StepStreams {
               e_bwd[pp::kStepChunks] = {};
 };
 StepStreams* step_streams() {
-  constexpr int kMaxDevices = 64;
   static std::mutex mu;
-  static StepStreams per_device[kMaxDevices];
+  static StepStreams per_device[pp::kMaxDevices];
   int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= pp::kMaxDevices) return nullptr;
   std::lock_guard<std::mutex> lock(mu);
   StepStreams& st = per_device[dev];
   if (!st.up) {

@@ -739,9 +739,11 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
                          const CUtensorMap& tv, const CUtensorMap& tdo, const CUtensorMap& tdq,
                          const BwdParams& prm, bool dq_cleared, cudaStream_t stream,
                          int* launches) {
-  static bool configured = false;
+  static DeviceSetup setup[kMaxDevices];
+  DeviceSetup* dev = device_setup(setup);
+  if (!dev) return cudaErrorInvalidDevice;
   auto kern = prm.dq_sem ? bwd_kernel<D, true> : bwd_kernel<D, false>;
-  if (!configured) {
+  if (!dev->configured) {
     cudaError_t e = cudaFuncSetAttribute(bwd_kernel<D, false>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          BwdSmem<D>::kTotal);
@@ -749,7 +751,7 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
       e = cudaFuncSetAttribute(bwd_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                BwdSmem<D>::kTotal);
     if (e != cudaSuccess) return e;
-    configured = true;
+    dev->configured = true;
   }
   const pp_problem& pb = plan->prob;
   const size_t T = pb.total_tokens, Hq = pb.num_q_heads;
@@ -765,13 +767,7 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
     bwd_preprocess_kernel<D, true><<<pre_blocks, 256, 0, stream>>>(
         static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse,
         const_cast<float*>(prm.delta), const_cast<float*>(prm.lse2), prm.dq_acc, int(T), int(Hq));
-  static int num_sms = 0;
-  if (!num_sms) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-      num_sms = 148;
-  }
+  const int num_sms = dev->num_sms;
   const long long units = (long long)plan->max_tiles * pb.num_kv_heads;
   dim3 grid(unsigned(std::min<long long>(units, num_sms)));
   ProfileEvents& ev = profile_events();
@@ -845,7 +841,6 @@ static __device__ __align__(256) unsigned char g_static_bwd_scratch[kStaticScrat
 // In host code `g_static_bwd_scratch` is only a stand-in for the symbol, not a device
 // address, so the address is looked up once per device (with that device current) and kept.
 static cudaError_t static_scratch_address(void** out) {
-  constexpr int kMaxDevices = 64;
   static std::mutex mu;
   static void* ptrs[kMaxDevices] = {};
   int dev = -1;

@@ -608,19 +608,17 @@ namespace {
 template <int D>
 cudaError_t launch_fwd_t(const pp_plan* plan, const CUtensorMap& tq, const CUtensorMap& tk,
                          const CUtensorMap& tv, const FwdParams& prm, cudaStream_t stream) {
-  static bool configured = false;
-  static int num_sms = 0;
+  static DeviceSetup setup[kMaxDevices];
+  DeviceSetup* dev = device_setup(setup);
+  if (!dev) return cudaErrorInvalidDevice;
   auto kern = fwd_kernel<D>;
-  if (!configured) {
+  if (!dev->configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          FwdSmem<D>::kTotal);
     if (e != cudaSuccess) return e;
-    int dev = 0;
-    cudaGetDevice(&dev);
-    e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return e;
-    configured = true;
+    dev->configured = true;
   }
+  const int num_sms = dev->num_sms;
   const pp_problem& pb = plan->prob;
   const int r = pb.num_q_heads / pb.num_kv_heads;
   const long long units = (long long)plan->max_tiles * pb.num_kv_heads * ((r + 1) / 2);

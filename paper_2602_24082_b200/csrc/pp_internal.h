@@ -165,6 +165,25 @@ inline StepArena step_arena_layout(const pp_problem& p) {
   return a;
 }
 
+// Per-device launch state of a kernel family: the opt-in to large dynamic shared memory is a
+// per-device function attribute, and the SM count differs between devices, so a process that
+// drives several GPUs must set up each of them.
+constexpr int kMaxDevices = 64;
+struct DeviceSetup {
+  bool configured = false;
+  int num_sms = 0;
+};
+// Entry for the current device in `table` (kMaxDevices entries), or null.
+inline DeviceSetup* device_setup(DeviceSetup* table) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  DeviceSetup* d = table + dev;
+  if (!d->num_sms &&
+      cudaDeviceGetAttribute(&d->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return nullptr;
+  return d;
+}
+
 // Optional event pairs around the forward kernel and the backward main kernel.
 struct ProfileEvents {
   bool on = false;
