@@ -249,6 +249,11 @@ int pp_last_launch_count(void);
  * Same layouts and errors as the calls above.
  */
 int pp_step_host_arena_bytes(const pp_problem* problem, size_t* arena_bytes);
+/* The runs pp_attn_step_host cuts `problem` into (host only, no device work): run c holds
+ * groups [group_begin[c], group_begin[c+1]) = tokens [token_begin[c], token_begin[c+1]).
+ * Both arrays must hold 9 entries. */
+int pp_step_host_runs(const pp_problem* problem, int32_t* num_runs, int32_t* group_begin,
+                      int32_t* token_begin);
 int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_k, const void* h_v,
                       const void* h_do, float softmax_scale, void* h_o, float* h_lse, void* h_dq,
                       void* h_dk, void* h_dv, void* d_arena, size_t arena_bytes,

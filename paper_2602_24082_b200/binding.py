@@ -22,7 +22,7 @@ _lib: Optional[ctypes.CDLL] = None
 
 EXPORTS = ["pp_plan_workspace_bytes", "pp_build_plan", "pp_plan_status", "pp_destroy_plan",
            "pp_plan_max_tiles", "pp_plan_read", "pp_attn_fwd", "pp_attn_bwd",
-           "pp_last_launch_count", "pp_error_string", "pp_step_host_arena_bytes",
+           "pp_last_launch_count", "pp_error_string", "pp_step_host_arena_bytes", "pp_step_host_runs",
            "pp_attn_step_host", "pp_profile_enable", "pp_profile_read",
            "pp_attn_bwd_noalloc", "pp_attn_bwd_noalloc_max_bytes", "pp_plan_read_bwd_units",
            "pp_plan_read_bwd_tiles", "pp_attn_bwd_deterministic",
@@ -77,6 +77,7 @@ def lib() -> ctypes.CDLL:
         L.pp_build_rows_workspace_bytes.argtypes = [ctypes.c_int32, vp]
         L.pp_build_rows.argtypes = [ctypes.c_int32, ctypes.c_int32, vp, vp, vp, ctypes.c_int32, vp, sz] + [vp] * 10
         L.pp_step_host_arena_bytes.argtypes = [vp, vp]
+        L.pp_step_host_runs.argtypes = [vp, vp, vp, vp]
         L.pp_attn_step_host.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp, sz, vp]
         L.pp_attn_bwd_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
         L.pp_attn_bwd_noalloc_max_bytes.argtypes = [vp]
@@ -345,6 +346,15 @@ def pp_step_host_arena_bytes(problem: _Problem) -> int:
     _check(lib().pp_step_host_arena_bytes(ctypes.byref(problem), ctypes.byref(n)),
            "pp_step_host_arena_bytes")
     return n.value
+
+
+def pp_step_host_runs(problem: _Problem) -> Tuple[np.ndarray, np.ndarray]:
+    """(group_begin, token_begin) of the runs pp_attn_step_host cuts the problem into."""
+    n = ctypes.c_int32(0)
+    gb, tb = np.zeros(9, dtype=np.int32), np.zeros(9, dtype=np.int32)
+    _check(lib().pp_step_host_runs(ctypes.byref(problem), ctypes.byref(n), gb.ctypes.data,
+                                   tb.ctypes.data), "pp_step_host_runs")
+    return gb[:n.value + 1], tb[:n.value + 1]
 
 
 class HostStep:

@@ -455,6 +455,12 @@ std::vector<StepChunk> cut_step(const pp_problem& p, int want) {
   return out;
 }
 
+// A run below a quarter MiB of input is all launch overhead: fewer runs then.
+int step_runs_wanted(const pp_problem& p) {
+  const size_t in_bytes = size_t(p.total_tokens) * (p.num_q_heads + p.num_kv_heads) * p.head_dim * 4;
+  return int(std::min<size_t>(pp::kStepChunks, std::max<size_t>(1, in_bytes >> 18)));
+}
+
 // Places the chunks' private blocks; false if they do not fit the arena's regions.
 bool place_step(std::vector<StepChunk>& chunks, const pp::StepArena& a, size_t heads_q) {
   size_t po = a.plan, so = a.scratch, lo = a.lse;
@@ -471,6 +477,30 @@ bool place_step(std::vector<StepChunk>& chunks, const pp::StepArena& a, size_t h
   return po <= a.scratch && so <= a.total && lo <= a.dq;
 }
 }  // namespace
+
+int pp_step_host_runs(const pp_problem* problem, int32_t* num_runs, int32_t* group_begin,
+                      int32_t* token_begin) {
+  int rc = check_problem_shape(problem);
+  if (rc) return rc;
+  if (problem->desc_on_device || !num_runs || !group_begin || !token_begin)
+    return PP_ERR_INVALID_ARG;
+  if (!problem->row_group_off || !problem->grp_prompt_len || !problem->grp_resp_off ||
+      !problem->resp_len)
+    return PP_ERR_INVALID_ARG;
+  rc = check_host_descriptors(problem);
+  if (rc) return rc;
+  const std::vector<StepChunk> chunks = cut_step(*problem, step_runs_wanted(*problem));
+  int g = 0;
+  for (size_t c = 0; c < chunks.size(); ++c) {
+    group_begin[c] = g;
+    token_begin[c] = int32_t(chunks[c].t0);
+    g += chunks[c].prob.num_groups;
+  }
+  group_begin[chunks.size()] = g;
+  token_begin[chunks.size()] = problem->total_tokens;
+  *num_runs = int32_t(chunks.size());
+  return PP_OK;
+}
 
 int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_k, const void* h_v,
                       const void* h_do, float softmax_scale, void* h_o, float* h_lse, void* h_dq,
@@ -501,10 +531,7 @@ int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_
   // inputs of run c+1 go up and the results of run c-1 come down (two copy engines, opposite
   // directions) while the kernels of run c execute.  Inside a run dO still goes up behind
   // the forward and O / LSE come down behind the backward.
-  // A run below a quarter MiB of input is all launch overhead: fewer runs then.
-  const size_t in_bytes = T * (Hq + Hkv) * D * 4;
-  const int want = int(std::min<size_t>(pp::kStepChunks, std::max<size_t>(1, in_bytes >> 18)));
-  std::vector<StepChunk> chunks = cut_step(*problem, want);
+  std::vector<StepChunk> chunks = cut_step(*problem, step_runs_wanted(*problem));
   if (!place_step(chunks, a, Hq)) {
     chunks = cut_step(*problem, 1);
     if (!place_step(chunks, a, Hq)) return PP_ERR_WORKSPACE_TOO_SMALL;

@@ -109,3 +109,37 @@ def test_binding_fails_loudly_without_gpu():
         pytest.skip("GPU present")
     with pytest.raises(RuntimeError):
         B.plan_for(W.config0())
+
+
+def _runs(w):
+    problem, _keep = B.make_problem(w.descriptors(), w.num_q_heads, w.num_kv_heads, w.head_dim,
+                                    w.total_tokens)
+    return B.pp_step_host_runs(problem)
+
+
+def test_host_step_runs_partition_the_groups(lib):
+    """The host step is cut at group boundaries into at most eight runs of about equal token
+    counts; runs are non-empty, contiguous and cover everything; tiny problems stay whole."""
+    rows = [[(50 + 13 * i, (20 + i, 7 * (i % 4) + 1)), (9 + i, (30,))] for i in range(11)]
+    w = W.Workload("runs", rows, 8, 2, 128, seed=1)
+    gb, tb = _runs(w)
+    rgo, gpl, gro, rl = w.descriptors()
+    glen = np.array([gpl[g] + rl[gro[g]:gro[g + 1]].sum() for g in range(len(gpl))])
+    gstart = np.concatenate([[0], np.cumsum(glen)])
+    assert len(gb) - 1 == 8 and gb[0] == 0 and gb[-1] == len(gpl) and (np.diff(gb) >= 1).all()
+    assert tb.tolist() == gstart[gb].tolist() and tb[-1] == w.total_tokens
+    # balance: no run exceeds the ideal share by more than the longest group
+    assert np.diff(tb).max() <= w.total_tokens / 8 + glen.max()
+    # fewer groups than runs: one group per run
+    w3 = W.Workload("runs3", [[(300, (140, 77))], [(64, (200, 1))], [(129, (640,))]], 4, 2, 128, seed=2)
+    gb, tb = _runs(w3)
+    assert gb.tolist() == [0, 1, 2, 3]
+    # under a quarter MiB of input per run: fewer runs (here: one)
+    tiny = W.Workload("tiny", [[(5, (2, 4)), (3, (1,))], [(3, (1, 2))]], 2, 1, 64, seed=3)
+    gb, tb = _runs(tiny)
+    assert gb.tolist() == [0, 3] and tb.tolist() == [0, tiny.total_tokens]
+    # one very long group among short ones keeps every later run non-empty
+    lop = W.Workload("lop", [[(1, (1,))], [(900, (300, 300))], [(2, (1, 1))], [(1, (2,))],
+                             [(5, (5,))], [(400, (1,))]], 16, 2, 128, seed=4)
+    gb, tb = _runs(lop)
+    assert gb[0] == 0 and gb[-1] == 6 and (np.diff(gb) >= 1).all() and (np.diff(tb) >= 1).all()
