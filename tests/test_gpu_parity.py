@@ -71,6 +71,8 @@ RAGGED = [
     # whole responses, responses of one token, segment boundaries on and next to tile edges
     ("d64-many-short-responses", [[(100, (7, 1, 30, 1, 1, 64, 2, 90, 13))]], 2, 1, 64),
     ("d128-aligned-and-off-by-one", [[(128, (128, 127, 129)), (127, (1, 128)), (129, (130,))]], 2, 2, 128),
+    # a token's heads span 16 KB: the backward's preprocess walks memory order from there on
+    ("d128-wide-heads", [[(70, (33, 129))], [(5, (64,))]], 64, 16, 128),
 ]
 
 
