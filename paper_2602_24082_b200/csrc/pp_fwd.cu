@@ -480,7 +480,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           xb[half] = mx;
           named_barrier_sync(bar_id, 64);
           const float m_new = fmaxf(m_used, fmaxf(mx, xb[half ^ 1]) * prm.scale_log2);
-          const bool need = (m_new - m_used) > kRescaleThreshold;
+          // Rows past the tile's end hold whatever follows in memory: they must not steer the
+          // warp-wide decision, or a row's rounding would depend on its neighbours' data.
+          const bool need = row < u_len && (m_new - m_used) > kRescaleThreshold;
           if (!__any_sync(0xffffffffu, need)) break;  // same rows, same values in the partner warp
           const float alpha = ex2(m_used - m_new);
           wait_bar(bar(kODone + s), (tcS - 1) & 1, abort_flag, prm.header, 42 + s);

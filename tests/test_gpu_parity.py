@@ -84,6 +84,50 @@ def test_ragged_shapes(name, rows, hq, hkv, d, desc_on_device):
     check_against_oracle(w, tens, _run_gpu(w, tens, desc_on_device, for_backward=desc_on_device))
 
 
+def _random_workload(seed):
+    """Seeded random structure: 1-3 rows of 1-3 groups, 1-5 responses each, lengths drawn so
+    that segment ends fall before, on and after tile boundaries; random GQA ratio (odd ones
+    included) and head size."""
+    rng = np.random.default_rng(seed)
+    pick = lambda: int(rng.choice([1, 2, 17, 63, 64, 65, 127, 128, 129, 200, 257]))
+    rows = [[(pick(), tuple(pick() for _ in range(rng.integers(1, 6))))
+             for _ in range(rng.integers(1, 4))] for _ in range(rng.integers(1, 4))]
+    hkv = int(rng.choice([1, 2, 3]))
+    r = int(rng.choice([1, 2, 3, 4, 5]))
+    d = int(rng.choice([64, 128]))
+    return W.Workload(f"random{seed}", rows, hkv * r, hkv, d, seed=1000 + seed)
+
+
+@pytest.mark.parametrize("seed", range(48))
+def test_random_structures(seed):
+    """Oracle parity on random structures; every other one also through the host step and
+    the deterministic backward, which must agree with the default path (O, LSE, dK, dV bit
+    for bit)."""
+    from paper_2602_24082_b200 import binding as B
+    w = _random_workload(seed)
+    tens = w.tensors()
+    gpu = _run_gpu(w, tens, desc_on_device=bool(seed & 1), for_backward=bool(seed & 2))
+    check_against_oracle(w, tens, gpu)
+    if seed % 2 == 0:
+        hs = B.HostStep(w)
+        hs(*[t.contiguous().pin_memory() for t in tens])
+        torch.cuda.synchronize()
+        got = [x.float().numpy().astype(np.float64) for x in (hs.o, hs.lse, hs.dq, hs.dk, hs.dv)]
+        for i in (0, 1, 3, 4):
+            assert np.array_equal(got[i], gpu[i])
+        assert _rel_l2(got[2], gpu[2]) < 1e-3
+        q, k, v, do = (x.cuda() for x in tens)
+        plan = B.plan_for(w)
+        o, lse = B.pp_attn_fwd(plan, q, k, v, w.softmax_scale)
+        runs = [B.pp_attn_bwd(plan, q, k, v, o, lse, do, w.softmax_scale, deterministic=True)
+                for _ in range(2)]
+        torch.cuda.synchronize()
+        assert plan.status() == (0, 0)
+        for a, b in zip(*runs):
+            assert torch.equal(a, b)
+        assert _rel_l2(runs[0][0].float().cpu().numpy().astype(np.float64), gpu[2]) < 1e-3
+
+
 def _subset_parity(w, row_ids, kv_heads):
     """Run the GPU on the whole workload, compare an independent sub-problem with the oracle."""
     tens = w.tensors()
