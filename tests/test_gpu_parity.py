@@ -84,27 +84,13 @@ def test_ragged_shapes(name, rows, hq, hkv, d, desc_on_device):
     check_against_oracle(w, tens, _run_gpu(w, tens, desc_on_device, for_backward=desc_on_device))
 
 
-def _random_workload(seed):
-    """Seeded random structure: 1-3 rows of 1-3 groups, 1-5 responses each, lengths drawn so
-    that segment ends fall before, on and after tile boundaries; random GQA ratio (odd ones
-    included) and head size."""
-    rng = np.random.default_rng(seed)
-    pick = lambda: int(rng.choice([1, 2, 17, 63, 64, 65, 127, 128, 129, 200, 257]))
-    rows = [[(pick(), tuple(pick() for _ in range(rng.integers(1, 6))))
-             for _ in range(rng.integers(1, 4))] for _ in range(rng.integers(1, 4))]
-    hkv = int(rng.choice([1, 2, 3]))
-    r = int(rng.choice([1, 2, 3, 4, 5]))
-    d = int(rng.choice([64, 128]))
-    return W.Workload(f"random{seed}", rows, hkv * r, hkv, d, seed=1000 + seed)
-
-
 @pytest.mark.parametrize("seed", range(48))
 def test_random_structures(seed):
     """Oracle parity on random structures; every other one also through the host step and
     the deterministic backward, which must agree with the default path (O, LSE, dK, dV bit
     for bit)."""
     from paper_2602_24082_b200 import binding as B
-    w = _random_workload(seed)
+    w = W.random_structure(seed)
     tens = w.tensors()
     gpu = _run_gpu(w, tens, desc_on_device=bool(seed & 1), for_backward=bool(seed & 2))
     check_against_oracle(w, tens, gpu)

@@ -25,6 +25,12 @@ def _global_mask(w):
     return m
 
 
+@pytest.mark.parametrize("seed", range(24))
+def test_plan_matches_dense_mask_on_random_structures(seed):
+    test_plan_matches_dense_mask(W.random_structure(seed), desc_on_device=bool(seed & 1))
+    test_backward_units_order(W.random_structure(seed))
+
+
 @pytest.mark.parametrize("w", CASES, ids=lambda w: w.name)
 @pytest.mark.parametrize("desc_on_device", [False, True], ids=["hostdesc", "devdesc"])
 def test_plan_matches_dense_mask(w, desc_on_device):
