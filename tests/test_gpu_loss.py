@@ -14,7 +14,7 @@ CASES = [
     W.Workload("single", [[(97, (64,)), (128, (128, 128, 7, 9, 40))], [(700, (1, 1))]], 2, 2, 64, seed=5),
     W.config2(),
     W.config4(3),
-]
+] + [W.random_structure(s) for s in range(8)]
 
 
 @pytest.mark.parametrize("w", CASES, ids=lambda w: w.name)

@@ -12,7 +12,7 @@ CASES = [
     W.config0(),
     W.Workload("ragged", [[(257, (5, 128, 31))], [(1, (1, 300))]], 4, 2, 128, seed=4),
     W.Workload("groups", [[(97, (64, 200)), (128, (128, 128)), (3, (2, 1))], [(700, (1,))]], 2, 2, 64, seed=5),
-]
+] + [W.random_structure(s) for s in range(8)]
 
 
 @pytest.mark.parametrize("w", CASES, ids=lambda w: w.name)
