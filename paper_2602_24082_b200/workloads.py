@@ -351,15 +351,19 @@ def unpacked(w: Workload, padded: bool = True):
     return uw, torch.tensor(gather, dtype=torch.long)
 
 
-def random_structure(seed: int) -> Workload:
+def random_structure(seed: int, long: bool = False) -> Workload:
     """Seeded random packing structure for tests: 1-3 rows of 1-3 groups with 1-5 responses
     each, lengths drawn so that segment ends fall before, on and after 128-token tile
-    boundaries; random GQA ratio (odd ones included) and head size."""
-    rng = np.random.default_rng(seed)
-    pick = lambda: int(rng.choice([1, 2, 17, 63, 64, 65, 127, 128, 129, 200, 257]))
+    boundaries; random GQA ratio (odd ones included) and head size.  ``long``: segments of up
+    to a dozen tiles (uniform lengths in [1, 1500])."""
+    rng = np.random.default_rng(seed + (7919 if long else 0))
+    if long:
+        pick = lambda: int(rng.integers(1, 1501))
+    else:
+        pick = lambda: int(rng.choice([1, 2, 17, 63, 64, 65, 127, 128, 129, 200, 257]))
     rows = [[(pick(), tuple(pick() for _ in range(rng.integers(1, 6))))
              for _ in range(rng.integers(1, 4))] for _ in range(rng.integers(1, 4))]
     hkv = int(rng.choice([1, 2, 3]))
     r = int(rng.choice([1, 2, 3, 4, 5]))
     d = int(rng.choice([64, 128]))
-    return Workload(f"random{seed}", rows, hkv * r, hkv, d, seed=1000 + seed)
+    return Workload(f"random{'-long' if long else ''}{seed}", rows, hkv * r, hkv, d, seed=1000 + seed)

@@ -124,6 +124,14 @@ def test_random_structures(seed):
         assert _rel_l2(runs[0][0].float().cpu().numpy().astype(np.float64), gpu[2]) < 1e-3
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_random_long_structures(seed):
+    """Segments of many tiles: the whole workload on the GPU, one KV-head group of it against
+    the oracle."""
+    w = W.random_structure(seed, long=True)
+    _subset_parity(w, list(range(len(w.rows))), [seed % w.num_kv_heads])
+
+
 def _subset_parity(w, row_ids, kv_heads):
     """Run the GPU on the whole workload, compare an independent sub-problem with the oracle."""
     tens = w.tensors()
