@@ -124,6 +124,29 @@ def test_random_structures(seed):
         assert _rel_l2(runs[0][0].float().cpu().numpy().astype(np.float64), gpu[2]) < 1e-3
 
 
+@pytest.mark.parametrize("d", [64, 128])
+def test_growing_scores_take_the_rescale_path(d):
+    """Later keys score far higher than earlier ones (queries and keys of later token ranges are
+    amplified), so a row's running maximum jumps by more than the forward's lazy-rescale
+    threshold (2^8) from one key tile to the next: the accumulator is rescaled and the tile
+    redone.  Unit-variance inputs almost never get there."""
+    w = W.Workload("growing", [[(600, (300, 200))], [(130, (270,))]], 4, 2, d, seed=77)
+    q, k, v, do = w.tensors()
+    T = w.total_tokens
+    gain = torch.ones(T)
+    for lo, hi, g in ((250, 420, 1.8), (420, 600, 2.6), (700, 900, 2.6), (950, 1100, 3.0), (1300, 1500, 2.4)):
+        gain[lo:hi] = g
+    q = (q.float() * gain[:, None, None]).to(q.dtype)
+    k = (k.float() * gain[:, None, None]).to(k.dtype)
+    tens = (q, k, v, do)
+    # the jumps are there: per 128-key tile, the row maxima of the scaled scores in log2 units
+    s = torch.einsum("qd,kd->qk", q[:600, 0].float(), k[:600, 0].float()) * w.softmax_scale * 1.4426950408889634
+    s = s.masked_fill(torch.triu(torch.ones(600, 600, dtype=torch.bool), 1), float("-inf"))
+    run = torch.cummax(torch.stack([s[:, i:i + 128].max(dim=1).values for i in range(0, 600, 128)], 1), 1).values
+    assert ((run[:, 1:] - run[:, :-1]) > 8).any(dim=1).float().mean() > 0.1   # of the prompt rows
+    check_against_oracle(w, tens, _run_gpu(w, tens, for_backward=True))
+
+
 @pytest.mark.parametrize("seed", range(6))
 def test_random_long_structures(seed):
     """Segments of many tiles: the whole workload on the GPU, one KV-head group of it against
