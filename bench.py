@@ -319,7 +319,7 @@ def run_ours(args):
     fwd_tflops = f_flops / (fwd_ms * 1e-3) / 1e12
     # DRAM bytes per launch of the backward main kernel from one ncu capture of this workload
     # (profiles/fwd_bwd_kernels_config1.md); other workloads have no capture -> null
-    traffic = 0.9644e9 if args.config == "config1" else None
+    traffic = 0.9708e9 if args.config == "config1" else None
     roofline = {"kernel": "bwd_kernel (dS/dQ/dK/dV main)", "bound": "tensor", "achieved": bwd_tflops,
                 "peak": peak, "unit": "TFLOP/s", "frac": bwd_tflops / peak, "peak_kind": f"of {peak_kind} (burst)",
                 "frac_of_sustained_peak": bwd_tflops / peak_sustained,
