@@ -191,6 +191,20 @@ def _group_parity(w, groups, kv_heads):
         assert bool(torch.isfinite(x).all())
 
 
+def test_element_offsets_beyond_32_bits():
+    """T * Hq * D above 2^31 elements (Q alone is 4.4 GB): every index computed in the kernels
+    and the launchers must be 64-bit.  Two small groups -- one sitting where the element offset
+    crosses 2^31, one at the very end -- are checked against the oracle on the highest KV head;
+    everything else must be finite."""
+    big = (8192, (4096, 4096))
+    rows = [[big] * 32 + [(520, (300, 200))] + [big] + [(77, (130, 1, 64))]]
+    w = W.Workload("beyond-32-bit", rows, 32, 8, 128, seed=91)
+    assert w.total_tokens * 32 * 128 > 2 ** 31
+    first_small = 32 * 16384
+    assert first_small * 32 * 128 <= 2 ** 31 < (first_small + 1020) * 32 * 128
+    _group_parity(w, [(0, 32), (0, 34)], [7])
+
+
 def _smallest_groups(w, n):
     sizes = sorted((p + sum(rs), ri, gi) for ri, row in enumerate(w.rows) for gi, (p, rs) in enumerate(row))
     return [(ri, gi) for (_, ri, gi) in sizes[:n]]

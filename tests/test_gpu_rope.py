@@ -74,3 +74,30 @@ def test_rope_then_attention_equals_unpacked_with_plain_positions():
         uo, _ = B.pp_attn_fwd(uplan, uq, uk, uv, w.softmax_scale)
         assert (uo.float() - o[idx].float()).abs().max().item() <= 2e-2
         off += r
+
+
+def test_rope_with_element_offsets_beyond_32_bits():
+    """Q of more than 2^31 elements: the rotation of the last tokens (largest offsets) and of
+    the tokens around the 2^31-element mark against the oracle, position ids bit for bit."""
+    from paper_2602_24082_b200 import binding as B
+    big = (8192, (4096, 4096))
+    w = W.Workload("beyond-32-bit", [[big] * 32 + [(520, (300, 200))] + [big] + [(77, (130, 1, 64))]],
+                   32, 8, 128, seed=91)
+    T = w.total_tokens
+    assert T * 32 * 128 > 2 ** 31
+    g = torch.Generator().manual_seed(5)
+    q = torch.randn(T, 32, 128, generator=g, dtype=torch.float32).to(torch.bfloat16)
+    k = torch.randn(T, 8, 128, generator=g, dtype=torch.float32).to(torch.bfloat16)
+    plan = B.plan_for(w, desc_on_device=True)
+    pos_gpu = B.pp_position_ids(plan).cpu().numpy()
+    pos = R.position_ids(w.rows)
+    assert np.array_equal(pos_gpu, pos)
+    qd, kd = q.cuda(), k.cuda()
+    B.pp_rope_qk(plan, qd, kd, 10000.0)
+    torch.cuda.synchronize()
+    for lo, hi in ((32 * 16384 - 64, 32 * 16384 + 600), (T - 300, T)):
+        for got, src in ((qd, q), (kd, k)):
+            ref = R.rope(src[lo:hi].double().numpy(), pos[lo:hi], 10000.0)
+            out = got[lo:hi].float().cpu().numpy().astype(np.float64)
+            assert np.abs(out - ref).max() <= 2e-2
+            assert np.linalg.norm(out - ref) / np.linalg.norm(ref) <= 4e-3
