@@ -262,8 +262,12 @@ int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_
 /*
  * Kernel timing for benchmarks.  pp_profile_enable(1) makes pp_attn_fwd / pp_attn_bwd record
  * CUDA events on the caller's stream directly around the forward kernel and around the
- * backward main kernel; pp_profile_read returns the two durations (ms) of the most recent
- * calls once that stream has been synchronised by the caller (PP_ERR_CUDA otherwise).
+ * backward main kernel; pp_profile_enable(2) only around the backward main kernel (every
+ * event between two kernels keeps the second from being queued behind the first, about 5 us
+ * each on a sub-millisecond step).  pp_profile_read returns the durations (ms) of the most
+ * recent calls once that stream has been synchronised by the caller (PP_ERR_CUDA otherwise;
+ * pass NULL for a duration that is not being recorded).  On a capturing stream the records
+ * become nodes of the graph and mark the events at every replay.
  * pp_profile_enable(0) releases the events.  One set of events per process, created on the
  * device that is current at pp_profile_enable(1): profile one device at a time.
  */

@@ -394,15 +394,23 @@ class HostStep:
         return self.o, self.lse, self.dq, self.dk, self.dv
 
 
-def pp_profile_enable(on: bool):
-    _check(lib().pp_profile_enable(1 if on else 0), "pp_profile_enable")
+def pp_profile_enable(on, backward_only: bool = False):
+    """Kernel event timing: both main kernels, or only the backward main kernel."""
+    global _profile_fwd
+    mode = 0 if not on else (2 if backward_only else 1)
+    _check(lib().pp_profile_enable(mode), "pp_profile_enable")
+    _profile_fwd = mode == 1
 
 
-def pp_profile_read() -> Tuple[float, float]:
-    """(forward kernel ms, backward main kernel ms) of the latest calls; sync the stream first."""
+_profile_fwd = False
+
+
+def pp_profile_read() -> Tuple[Optional[float], float]:
+    """(forward kernel ms or None, backward main kernel ms) of the latest calls; sync the stream first."""
     a, b = ctypes.c_float(0), ctypes.c_float(0)
-    _check(lib().pp_profile_read(ctypes.byref(a), ctypes.byref(b)), "pp_profile_read")
-    return a.value, b.value
+    _check(lib().pp_profile_read(ctypes.byref(a) if _profile_fwd else None, ctypes.byref(b)),
+           "pp_profile_read")
+    return (a.value if _profile_fwd else None), b.value
 
 
 def pp_last_launch_count() -> int:

@@ -612,7 +612,10 @@ int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_
   return joined ? PP_OK : PP_ERR_CUDA;
 }
 
-int pp_profile_enable(int on) { return pp::profile_enable(on != 0) ? PP_OK : PP_ERR_CUDA; }
+int pp_profile_enable(int on) {
+  if (on < 0 || on > 2) return PP_ERR_INVALID_ARG;
+  return pp::profile_enable(on) ? PP_OK : PP_ERR_CUDA;
+}
 
 int pp_profile_read(float* fwd_kernel_ms, float* bwd_main_kernel_ms) {
   return pp::profile_read(fwd_kernel_ms, bwd_main_kernel_ms) ? PP_OK : PP_ERR_CUDA;

@@ -793,10 +793,10 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
   const long long units = (long long)plan->max_tiles * pb.num_kv_heads;
   dim3 grid(unsigned(std::min<long long>(units, num_sms)));
   ProfileEvents& ev = profile_events();
-  if (ev.on) cudaEventRecord(ev.bwd0, stream);
+  if (ev.on) profile_record(ev.bwd0, stream);
   kern<<<grid, kBwdThreads, BwdSmem<D>::kTotal, stream>>>(tq, tk, tv, tdo, tdq, prm);
   if (ev.on) {
-    cudaEventRecord(ev.bwd1, stream);
+    profile_record(ev.bwd1, stream);
     ev.bwd_valid = true;
   }
   const size_t n4 = T * Hq * D / 4;

@@ -626,10 +626,10 @@ cudaError_t launch_fwd_t(const pp_plan* plan, const CUtensorMap& tq, const CUten
   const long long units = (long long)plan->max_tiles * pb.num_kv_heads * ((r + 1) / 2);
   dim3 grid(unsigned(std::min<long long>(units, num_sms)));
   ProfileEvents& ev = profile_events();
-  if (ev.on) cudaEventRecord(ev.fwd0, stream);
+  if (ev.on && ev.fwd_on) profile_record(ev.fwd0, stream);
   kern<<<grid, kFwdThreads, FwdSmem<D>::kTotal, stream>>>(tq, tk, tv, prm);
-  if (ev.on) {
-    cudaEventRecord(ev.fwd1, stream);
+  if (ev.on && ev.fwd_on) {
+    profile_record(ev.fwd1, stream);
     ev.fwd_valid = true;
   }
   return cudaGetLastError();

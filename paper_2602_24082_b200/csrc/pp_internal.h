@@ -187,11 +187,21 @@ inline DeviceSetup* device_setup(DeviceSetup* table) {
 // Optional event pairs around the forward kernel and the backward main kernel.
 struct ProfileEvents {
   bool on = false;
+  bool fwd_on = false;  // forward events wanted too (mode 1); mode 2 times the backward only
   cudaEvent_t fwd0 = nullptr, fwd1 = nullptr, bwd0 = nullptr, bwd1 = nullptr;
   bool fwd_valid = false, bwd_valid = false;
 };
 ProfileEvents& profile_events();
-bool profile_enable(bool on);
+// Records a profiling event.  On a capturing stream the record becomes a node of the graph
+// that marks the event at every replay (an ordinary record would only order the capture).
+inline void profile_record(cudaEvent_t ev, cudaStream_t stream) {
+  cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(stream, &st) == cudaSuccess && st == cudaStreamCaptureStatusActive)
+    cudaEventRecordWithFlags(ev, stream, cudaEventRecordExternal);
+  else
+    cudaEventRecord(ev, stream);
+}
+bool profile_enable(int mode);
 bool profile_read(float* fwd_ms, float* bwd_ms);
 
 // launchers (defined in the .cu files); all return a cudaError_t

@@ -438,13 +438,19 @@ ProfileEvents& profile_events() {
   return ev;
 }
 
-bool profile_enable(bool on) {
+bool profile_enable(int mode) {
   ProfileEvents& ev = profile_events();
+  const bool on = mode != 0;
+  if (on && ev.on) {  // already on: only the choice of kernels can change
+    ev.fwd_on = mode == 1;
+    return true;
+  }
   if (on == ev.on) return true;
   if (on) {
     bool ok = cudaEventCreate(&ev.fwd0) == cudaSuccess && cudaEventCreate(&ev.fwd1) == cudaSuccess &&
               cudaEventCreate(&ev.bwd0) == cudaSuccess && cudaEventCreate(&ev.bwd1) == cudaSuccess;
     ev.on = ok;
+    ev.fwd_on = mode == 1;
     ev.fwd_valid = ev.bwd_valid = false;
     return ok;
   }

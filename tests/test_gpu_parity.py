@@ -398,3 +398,46 @@ def test_host_step_matches_the_device_path(w):
             assert np.array_equal(got[i], ref[i])
         assert _rel_l2(got[2], ref[2]) < 1e-3
     check_against_oracle(w, tens, tuple(got))
+
+
+def test_step_can_be_captured_in_a_cuda_graph():
+    """Plan building, forward and backward make no host synchronisation and no allocation, so
+    the three calls can be stream-captured; replays reproduce the eager results (O, LSE, dK,
+    dV bit for bit) also after the inputs have changed in place."""
+    from paper_2602_24082_b200 import binding as B
+    w = W.Workload("graph", [[(300, (140, 77))], [(64, (200, 1))]], 4, 2, 128, seed=41)
+    q, k, v, do = (x.cuda() for x in w.tensors())
+    desc = w.descriptors()
+    desc_dev = [torch.from_numpy(np.ascontiguousarray(a)).cuda() for a in desc]
+    problem, _keep = B.make_problem(desc, 4, 2, 128, w.total_tokens, desc_dev)
+    ws = torch.empty(B.pp_plan_workspace_bytes(problem)[0], dtype=torch.uint8, device="cuda")
+    o, lse = torch.empty_like(q), torch.empty(4, w.total_tokens, dtype=torch.float32, device="cuda")
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    hold = {}
+
+    def step():
+        plan = B.pp_build_plan(desc, 4, 2, 128, w.total_tokens, "cuda:0", device_arrays=desc_dev, workspace=ws)
+        if "scratch" in hold:
+            plan._bwd_scratch = hold["scratch"]
+        B.pp_attn_fwd(plan, q, k, v, w.softmax_scale, o=o, lse=lse, for_backward=True)
+        B.pp_attn_bwd(plan, q, k, v, o, lse, do, w.softmax_scale, d_q=dq, d_k=dk, d_v=dv)
+        hold["scratch"], hold["plan"] = plan.bwd_scratch(), plan
+
+    step()                      # first calls configure the kernels: not inside a capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for scale_inputs in (1.0, 0.5):
+        q.mul_(scale_inputs)
+        step()
+        torch.cuda.synchronize()
+        want = [x.clone() for x in (o, lse, dk, dv, dq)]
+        for x in (o, lse, dk, dv, dq):
+            x.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert hold["plan"].status() == (0, 0)
+        for got, ref in zip((o, lse, dk, dv), want):
+            assert torch.equal(got, ref)
+        assert _rel_l2(dq.float().cpu().numpy(), want[4].float().cpu().numpy()) < 1e-3
