@@ -381,52 +381,72 @@ __global__ void __launch_bounds__(1024) plan_fused_kernel(PlanPtrs p) {
     const Tile tl = p.tiles[t];
     for (int i = tid & 31; i < tl.len; i += 32) p.key_end[tl.start + i] = tl.vis_end;
   }
-  // longest-work-first orders by rank counting, and the work of each backward tile's group
-  for (int t = tid; t < n; t += nthr) {
+  // Longest-work-first orders by rank counting, and the work of each backward tile's group.
+  // One warp per tile: the lanes stride over the other tiles and the partial counts are
+  // summed with shuffles (a thread per tile would walk the whole list alone, a few
+  // microseconds of dependent shared-memory reads per pass on a 100-tile plan).
+  const int lane = tid & 31, wid = tid >> 5, nwarp = nthr >> 5;
+  auto warp_sum = [](int x) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) x += __shfl_xor_sync(0xffffffffu, x, d);
+    return x;
+  };
+  for (int t = wid; t < n; t += nwarp) {
     const int wf = s_wf[t];
     int rf = 0;
-    for (int u = 0; u < n; ++u) {
+    for (int u = lane; u < n; u += 32) {
       const int of = s_wf[u];
       rf += (of > wf) || (of == wf && u < t);
     }
-    p.fwd_order[rf] = t;
+    rf = warp_sum(rf);
+    if (lane == 0) p.fwd_order[rf] = t;
   }
-  for (int t = tid; t < nb; t += nthr) {
+  for (int t = wid; t < nb; t += nwarp) {
     const int wb = s_wb[t], gs = s_gs[t];
     int rb = 0, gw = 0;
-    for (int u = 0; u < nb; ++u) {
+    for (int u = lane; u < nb; u += 32) {
       const int ob = s_wb[u];
       rb += (ob > wb) || (ob == wb && u < t);
       gw += (s_gs[u] == gs) ? ob : 0;
     }
-    p.bwd_order[rb] = t;
-    p.tile_gwork[t] = gw;
-    s_gw[t] = gw;
+    rb = warp_sum(rb);
+    gw = warp_sum(gw);
+    if (lane == 0) {
+      p.bwd_order[rb] = t;
+      p.tile_gwork[t] = gw;
+      s_gw[t] = gw;
+    }
   }
   __syncthreads();
-  for (int t = tid; t < nb; t += nthr) {
+  for (int t = wid; t < nb; t += nwarp) {
     const int gs = s_gs[t], gw = s_gw[t];
     int rest = 0;  // tiles of this group and of the groups that come later
-    for (int u = 0; u < nb; ++u) {
+    for (int u = lane; u < nb; u += 32) {
       const int ogs = s_gs[u], ow = s_gw[u];
       rest += (ogs == gs) || (ow < gw) || (ow == gw && ogs > gs);
     }
-    const int sg = (p.Hkv * rest - 1) / kSuperGroupUnits;
-    p.tile_sgroup[t] = sg;
-    s_sg[t] = uint16_t(sg);
+    rest = warp_sum(rest);
+    if (lane == 0) {
+      const int sg = (p.Hkv * rest - 1) / kSuperGroupUnits;
+      p.tile_sgroup[t] = sg;
+      s_sg[t] = uint16_t(sg);
+    }
   }
   __syncthreads();
-  for (int t = tid; t < nb; t += nthr) {
+  for (int t = wid; t < nb; t += nwarp) {
     const int sg = s_sg[t], wb = s_wb[t];
     int pos = 0, dpos = 0;
-    for (int u = 0; u < nb; ++u) {
+    for (int u = lane; u < nb; u += 32) {
       const int osg = s_sg[u], ob = s_wb[u];
       pos += (osg > sg) || (osg == sg && ((ob > wb) || (ob == wb && u < t)));
       dpos += (osg > sg) || (osg == sg && u < t);
     }
-    for (int kvh = 0; kvh < p.Hkv; ++kvh) {
+    pos = warp_sum(pos);
+    dpos = warp_sum(dpos);
+    // ascending tiles inside a super-group for the deterministic backward
+    for (int kvh = lane; kvh < p.Hkv; kvh += 32) {
       p.bwd_units[p.Hkv * pos + kvh] = (kvh << 24) | t;
-      p.bwd_units_det[p.Hkv * dpos + kvh] = (kvh << 24) | t;  // ascending tiles in a super-group
+      p.bwd_units_det[p.Hkv * dpos + kvh] = (kvh << 24) | t;
     }
   }
 }
