@@ -296,7 +296,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     int u = 0;
     if (lane == 0) {
       wait_bar(bar(kSchedEmpty + (n & 1)), ((n >> 1) & 1) ^ 1, abort_flag, prm.header, 90);
-      u = atomicAdd(&prm.header[kHdrBwdNext], 1);
+      // after a wait has given up, no more work is drawn: an out-of-range id ends every role
+      u = *abort_flag ? 0x7fffffff : atomicAdd(&prm.header[kHdrBwdNext], 1);
       sched[n & 1] = u;
       mbar_arrive(bar(kSchedFull + (n & 1)));
     }
@@ -329,7 +330,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         }
       }
       QIter qi;
-      for (int it = 0; it < un.n_it; ++it, ++qc, q_advance(qi, prm.Hq / prm.Hkv)) {
+      for (int it = 0; it < un.n_it && !*abort_flag; ++it, ++qc, q_advance(qi, prm.Hq / prm.Hkv)) {
         const QTile qt = q_tile_at(prm, un, qi);
         const uint32_t st = qc & 1, par = ((qc >> 1) & 1) ^ 1;
         // per-query statistics, fetched before the stage is known to be free;
@@ -716,6 +717,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 
   tc_fence_before();
   __syncthreads();
+  // After a wait that gave up, copies, reductions and MMAs issued without their barriers may
+  // still be in flight: give them time to land before shared and tensor memory are released.
+  if (*abort_flag)
+    for (int i = 0; i < 50; ++i) __nanosleep(1000);
   if (warp == 0) tmem_dealloc(tmem, kBwdTmemCols);
   if (tid == 0) {  // the last CTA to finish re-arms the unit counter for the next launch
     __threadfence();

@@ -167,7 +167,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   volatile int* sched = reinterpret_cast<volatile int*>(gbase + L::kSched);
   auto fetch_unit = [&](uint32_t n, Unit& un) -> bool {  // producer thread
     wait_bar(bar(kSchedEmptyF + (n & 1)), ((n >> 1) & 1) ^ 1, abort_flag, prm.header, 90);
-    const int u = atomicAdd(&prm.header[kHdrFwdNext], 1);
+    // after a wait has given up, no more work is drawn: the end marker goes out instead
+    const int u = *abort_flag ? 0x7fffffff : atomicAdd(&prm.header[kHdrFwdNext], 1);
     const bool ok = get_unit(prm, u, ntiles_total, un);
     volatile int* e = sched + (n & 1) * 8;
     e[0] = un.tile.start;
@@ -238,7 +239,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           ++vc;
         };
         load_k(0);
-        for (int j = 0; j < un.ntiles; ++j) {
+        for (int j = 0; j < un.ntiles && !*abort_flag; ++j) {
           if (j + 1 < un.ntiles) load_k(j + 1);
           load_v(j);
         }
@@ -574,6 +575,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 
   tc_fence_before();
   __syncthreads();
+  // After a wait that gave up, copies and MMAs issued without their barriers may still be in
+  // flight: give them time to land before the CTA's shared and tensor memory are released.
+  if (*abort_flag)
+    for (int i = 0; i < 50; ++i) __nanosleep(1000);
   if (warp == 0) tmem_dealloc(tmem, kFwdTmemCols);
   if (tid == 0) {  // the last CTA to finish re-arms the unit counter for the next launch
     __threadfence();
