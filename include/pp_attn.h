@@ -19,7 +19,8 @@
  *   Base pointers must be 16-byte aligned.  Inputs must be finite.
  *
  * All functions return 0 (PP_OK) or a negative pp_status; they never throw, exit or print.
- * Work is enqueued on the caller's stream; only pp_plan_status synchronises.
+ * Work is enqueued on the caller's stream; only pp_plan_status and the pp_plan_read* test
+ * accessors synchronise it.
  */
 #ifndef PP_ATTN_H_
 #define PP_ATTN_H_
@@ -49,7 +50,8 @@ enum pp_status {
 /*
  * Problem statement, in the paper's terms (Sec. 3.1 symbols): per group g one prompt of
  * length P_g (l_in) and n_g >= 1 responses of lengths R_{g,1..n_g} (l_resp^k).
- * Descriptor arrays are int32 and are read during pp_build_plan only.
+ * Descriptor arrays are int32 and are read by pp_build_plan only: host arrays during the call,
+ * device arrays by the plan kernels it enqueues (keep them unchanged until those have run).
  */
 typedef struct {
   int32_t num_rows;
