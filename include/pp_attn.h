@@ -248,7 +248,8 @@ int pp_last_launch_count(void);
  * d_arena is caller-owned device memory of at least pp_step_host_arena_bytes (256-byte
  * aligned); it holds the device copies, the plan workspaces and the backward scratch.
  * `problem` must have desc_on_device == 0; its descriptors are validated on the host first.
- * Same layouts and errors as the calls above.
+ * All calls on one device share the two side streams and their events: make them from one
+ * host thread at a time.  Same layouts and errors as the calls above.
  */
 int pp_step_host_arena_bytes(const pp_problem* problem, size_t* arena_bytes);
 /* The runs pp_attn_step_host cuts `problem` into (host only, no device work): run c holds
