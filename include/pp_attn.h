@@ -39,7 +39,7 @@ enum pp_status {
   PP_OK = 0,
   PP_ERR_INVALID_ARG = -1,         /* null pointer, non-positive length, non-monotone offsets,
                                       total_tokens mismatch, Hq % Hkv != 0 */
-  PP_ERR_UNSUPPORTED = -2,         /* head_dim not in {64, 128}; device is not sm_100 */
+  PP_ERR_UNSUPPORTED = -2,         /* head_dim not in {64, 128}; device is not compute capability 10.x */
   PP_ERR_WORKSPACE_TOO_SMALL = -3, /* plan workspace or scratch smaller than the size query says */
   PP_ERR_ALIGNMENT = -4,           /* a tensor base pointer is not 16-byte aligned */
   PP_ERR_CUDA = -5,                /* a CUDA runtime / driver call failed */
@@ -51,7 +51,9 @@ enum pp_status {
  * Problem statement, in the paper's terms (Sec. 3.1 symbols): per group g one prompt of
  * length P_g (l_in) and n_g >= 1 responses of lengths R_{g,1..n_g} (l_resp^k).
  * Descriptor arrays are int32 and are read by pp_build_plan only: host arrays during the call,
- * device arrays by the plan kernels it enqueues (keep them unchanged until those have run).
+ * device arrays by the first plan kernel it enqueues, which copies them into the workspace
+ * (keep them unchanged until that kernel has run; everything later -- the other plan kernels,
+ * pp_position_ids, pp_rope_qk, pp_preference_loss -- reads the copy).
  */
 typedef struct {
   int32_t num_rows;
@@ -89,10 +91,20 @@ int pp_plan_workspace_bytes(const pp_problem* problem, size_t* plan_bytes,
  * workspace: up to 7168 entries over the four arrays travel as the argument of a small kernel,
  * so the call never waits on the host for work already in `stream`; longer ones are copied
  * with cudaMemcpyAsync, which for pageable host memory does wait for the stream first.  The
- * host arrays may be changed or freed as soon as the call returns.
- * d_workspace must stay alive and untouched while the plan is used.  The plan is
- * immutable and can be reused by any number of pp_attn_fwd / pp_attn_bwd calls whose
- * tensors have the shapes stated in `problem`.
+ * host arrays may be changed or freed as soon as the call returns -- except page-locked arrays
+ * of more than 7168 entries, which the copy reads asynchronously: keep those unchanged until
+ * `stream` has reached the plan kernels.
+ * d_workspace must stay alive and untouched while the plan is used.  The plan's tables are
+ * fixed once built and serve any number of pp_attn_fwd / pp_attn_bwd calls whose tensors have
+ * the shapes stated in `problem`, with two pieces of mutable state to respect:
+ *  - the workspace holds the work counters the kernels draw their units from (re-armed by the
+ *    last CTA of each launch), so two forwards, or two backwards, on ONE plan must not overlap
+ *    on the GPU: order them on one stream (or by events); overlapping launches would each
+ *    process part of the work and leave outputs partly unwritten.  Build one plan per stream
+ *    for concurrent use.  A forward and a backward never share a counter.
+ *  - the host handle remembers which scratch buffer the latest pp_attn_fwd cleared for the next
+ *    pp_attn_bwd (see pp_attn_fwd): calls on one plan must come from one host thread at a time.
+ * Returns PP_ERR_UNSUPPORTED when the current device is not compute capability 10.x.
  */
 int pp_build_plan(const pp_problem* problem, void* d_workspace, size_t workspace_bytes,
                   pp_stream_t stream, pp_plan** out_plan);
@@ -173,8 +185,8 @@ int pp_attn_bwd_deterministic(const pp_plan* plan, const void* q, const void* k,
                               void* d_scratch, size_t scratch_bytes, pp_stream_t stream);
 
 /*
- * The step right before attention (Sec. 3.2: "position IDs help positional embeddings retain
- * their original positions").  pp_position_ids writes, per token, the position it would have
+ * The step right before attention (Sec. 3.2: every token keeps the position it has in its own
+ * unpacked sequence).  pp_position_ids writes, per token, the position it would have
  * in its own unpacked sequence (x, y^k): index inside the prompt for prompt tokens, P + index
  * inside the response for response tokens -- positions restart after the prompt for every
  * response.  pp_rope_qk applies the rotary embedding (rotate-half form, angle = position *
@@ -215,8 +227,10 @@ int pp_preference_loss(const pp_plan* plan, const float* token_logp, const float
  *    pp_attn_bwd_noalloc_max_bytes (32 MiB, i.e. about T * Hq * D <= 8.2 M elements);
  *    larger problems are rejected with PP_ERR_STATIC_SCRATCH_LIMIT and nothing is launched.
  *  - Cost: every GPU on which the library is loaded holds those 32 MiB until the process exits.
- *  - The first call on each device looks up the array's device address (with that device
- *    current).  Make that first call before any stream capture begins.
+ *  - The array used is the one on the device that holds the plan's workspace, and that device
+ *    must be the current device at the call (PP_ERR_INVALID_ARG otherwise: another device's
+ *    array is never handed to the kernels).  The first call on each device looks up the
+ *    array's device address.  Make that first call before any stream capture begins.
  *  - All calls on a device share the one array, and it keeps the previous call's contents.
  *    Each call clears the part that must start at zero (the dQ accumulator) and rewrites
  *    the rest, so back-to-back calls on ONE stream are safe; calls that can overlap on the
@@ -278,11 +292,12 @@ int pp_profile_enable(int on);
 int pp_profile_read(float* fwd_kernel_ms, float* bwd_main_kernel_ms);
 
 /*
- * Row builder: the step before the attention path (Sec. 2.3, applied together with preference
- * packing in Sec. 4.3).  Groups [prompt | responses] are ordered by total length, longest first
- * and ties in their original order ("batch sorting"), and consecutive groups of that order
- * are concatenated into rows of at most row_capacity tokens (packing "up to a maximum sequence
- * length": next fit).  All pointers are DEVICE pointers; everything runs on `stream`.
+ * Row builder: the step before the attention path (batch sorting and batch packing, Sec. 2.2;
+ * applied together with preference packing in Sec. 5.2, Table 2).  Groups [prompt | responses]
+ * are ordered by total length, longest first and ties in their original order (batch sorting),
+ * and consecutive groups of that order are concatenated into rows of at most row_capacity
+ * tokens (batch packing; next fit).  All pointers are DEVICE pointers; everything runs on
+ * `stream`.
  *   in : grp_prompt_len [G], grp_resp_off [G + 1], resp_len [N]        (int32, as in pp_problem)
  *   out: order [G]            original index of the group at each position of the new order
  *        row_group_off [G + 1], num_rows [1]   positions [off[r], off[r + 1]) form row r
@@ -303,6 +318,35 @@ int pp_build_rows(int32_t num_groups, int32_t num_responses, const int32_t* grp_
                   int32_t* row_group_off, int32_t* num_rows, int64_t* row_tokens,
                   int64_t* row_cost, int32_t* out_prompt_len, int32_t* out_resp_off,
                   int32_t* out_resp_len, int32_t* status, pp_stream_t stream);
+
+/*
+ * Rows -> data-parallel ranks (Sec. 2.2: batch sorting exists so that no rank waits for the
+ * one with the longest sequences; Sec. 5.2, Table 2, the run with sorting and packing both).
+ * Longest-processing-time assignment by attention cost: rows are taken in order of decreasing
+ * row_cost (ties: lower index first) and each goes to the rank whose cost so far is least
+ * (ties: lowest rank).  Every rank's total then stays within (mean + largest row cost).
+ * All pointers are DEVICE pointers; two small kernels on `stream`; nothing is allocated.
+ *   in : row_cost [num_rows] (int64; pp_build_rows' row_cost, or any non-negative cost)
+ *   out: order [num_rows]        rows in the order they were assigned
+ *        rank_of_row [num_rows]  rank that processes each row
+ *        rank_cost [num_ranks]   (int64) total cost per rank
+ * num_rows <= 65536, num_ranks <= 1024 (PP_ERR_UNSUPPORTED beyond); PP_ERR_INVALID_ARG,
+ * PP_ERR_CUDA.  The ranks themselves exchange nothing: each computes the same assignment from
+ * the same costs and processes its own rows.
+ */
+int pp_assign_rows(int32_t num_rows, const int64_t* row_cost, int32_t num_ranks, int32_t* order,
+                   int32_t* rank_of_row, int64_t* rank_cost, pp_stream_t stream);
+
+/*
+ * Test hook for the bounded waits (no counterpart in the paper).  Every wait inside the
+ * kernels polls a bounded number of times and then records kStatusWaitExpired (3) with the
+ * wait's site id in the plan's status word instead of spinning on.  This call runs that same
+ * wait routine in a one-thread kernel on a barrier nobody arrives at, with a limit of 4096
+ * polls and with no copy or MMA in flight, so the give-up path can be checked on a GPU without
+ * hanging anything: afterwards pp_plan_status reports status 3 / detail `site`, and the
+ * kernels of later calls on this plan return at once.  site >= 1.
+ */
+int pp_debug_expire_wait(const pp_plan* plan, int32_t site, pp_stream_t stream);
 
 const char* pp_error_string(int code);
 

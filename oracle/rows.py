@@ -1,16 +1,16 @@
 """Oracle for the row builder (test infrastructure: only tests, smoke() and the benchmark's CPU
 legs may import this package; the product path never does).
 
-The step before the attention path (paper Sec. 2.3 and 4.3): preference groups
+The step before the attention path (paper Sec. 2.2; used with preference packing in Sec. 5.2,
+Table 2): preference groups
 [prompt | responses] of varying length are put into rows of at most `capacity` tokens.
 
 Reading of the paper (it names the two techniques and gives no algorithm):
-  * batch sorting -- "grouping samples of similar lengths into the same batch": the groups
-    are ordered by total length (prompt + all responses), longest first; ties keep their
-    original order;
-  * packing -- "concatenates individual sequences in a sequence-wise manner up to a maximum
-    sequence length": consecutive groups of that order are concatenated into one row while
-    the row stays within `capacity` (next fit), so a row holds groups of similar length;
+  * batch sorting (samples of similar length share a batch): the groups are ordered by total
+    length (prompt + all responses), longest first; ties keep their original order;
+  * batch packing (sequences concatenated up to a length limit): consecutive groups of that
+    order are concatenated into one row while the row stays within `capacity` (next fit), so
+    a row holds groups of similar length;
   * rows therefore come out in decreasing length, and a data-parallel step takes consecutive
     rows, one per rank, which is what keeps the ranks' work similar; `row_cost` (visible
     query-key pairs, the attention cost of Sec. 3.2.1) is reported for that purpose.
@@ -86,3 +86,21 @@ def build_rows(grp_prompt_len, grp_resp_off, resp_len, capacity):
             "row_tokens": np.asarray(row_tokens, dtype=np.int64),
             "row_cost": np.asarray(row_cost, dtype=np.int64),
             "grp_prompt_len": i32(new_P), "grp_resp_off": i32(new_off), "resp_len": i32(new_R)}
+
+
+def assign_rows(row_cost, num_ranks):
+    """Rows -> data-parallel ranks (Sec. 2.2: sorting by length exists so that no rank waits for
+    the one holding the longest sequences).  Reading: longest-processing-time list scheduling
+    on the attention cost -- rows in order of decreasing cost (ties: lower index first), each
+    to the rank with the least total so far (ties: lowest rank).
+    Returns (order [rows], rank_of_row [rows], rank_cost [ranks])."""
+    cost = [int(c) for c in row_cost]
+    order = sorted(range(len(cost)), key=lambda r: (-cost[r], r))
+    load = [0] * num_ranks
+    rank_of_row = [0] * len(cost)
+    for r in order:
+        k = min(range(num_ranks), key=lambda i: (load[i], i))
+        rank_of_row[r] = k
+        load[k] += cost[r]
+    return (np.asarray(order, dtype=np.int32), np.asarray(rank_of_row, dtype=np.int32),
+            np.asarray(load, dtype=np.int64))

@@ -27,7 +27,8 @@ EXPORTS = ["pp_plan_workspace_bytes", "pp_build_plan", "pp_plan_status", "pp_des
            "pp_attn_bwd_noalloc", "pp_attn_bwd_noalloc_max_bytes", "pp_plan_read_bwd_units",
            "pp_plan_read_bwd_tiles", "pp_attn_bwd_deterministic",
            "pp_position_ids", "pp_rope_qk", "pp_preference_loss",
-           "pp_build_rows_workspace_bytes", "pp_build_rows"]
+           "pp_build_rows_workspace_bytes", "pp_build_rows", "pp_assign_rows",
+           "pp_debug_expire_wait"]
 
 
 class PPError(RuntimeError):
@@ -76,6 +77,8 @@ def lib() -> ctypes.CDLL:
         L.pp_attn_bwd_deterministic.argtypes = L.pp_attn_bwd.argtypes
         L.pp_build_rows_workspace_bytes.argtypes = [ctypes.c_int32, vp]
         L.pp_build_rows.argtypes = [ctypes.c_int32, ctypes.c_int32, vp, vp, vp, ctypes.c_int32, vp, sz] + [vp] * 10
+        L.pp_assign_rows.argtypes = [ctypes.c_int32, vp, ctypes.c_int32, vp, vp, vp, vp]
+        L.pp_debug_expire_wait.argtypes = [vp, ctypes.c_int32, vp]
         L.pp_step_host_arena_bytes.argtypes = [vp, vp]
         L.pp_step_host_runs.argtypes = [vp, vp, vp, vp]
         L.pp_attn_step_host.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -452,3 +455,25 @@ def pp_build_rows(grp_prompt_len: torch.Tensor, grp_resp_off: torch.Tensor, resp
     r = int(nrows.item())
     return {"order": order, "row_group_off": rgo[:r + 1], "row_tokens": rtok[:r], "row_cost": rcost[:r],
             "grp_prompt_len": oP, "grp_resp_off": ooff, "resp_len": orl, "status": (st[0], st[1])}
+
+
+def pp_assign_rows(row_cost: torch.Tensor, num_ranks: int):
+    """Rows -> data-parallel ranks by longest-processing-time assignment on the attention cost.
+    ``row_cost``: int64 DEVICE tensor [rows].  Returns device tensors (order [rows] int32,
+    rank_of_row [rows] int32, rank_cost [num_ranks] int64)."""
+    _chk(row_cost, (row_cost.numel(),), torch.int64, "row_cost")
+    dev, R = row_cost.device, int(row_cost.numel())
+    order = torch.empty(R, dtype=torch.int32, device=dev)
+    rank_of_row = torch.empty(R, dtype=torch.int32, device=dev)
+    rank_cost = torch.empty(int(num_ranks), dtype=torch.int64, device=dev)
+    with torch.cuda.device(dev):
+        _check(lib().pp_assign_rows(R, row_cost.data_ptr(), int(num_ranks), order.data_ptr(),
+                                    rank_of_row.data_ptr(), rank_cost.data_ptr(), _stream()),
+               "pp_assign_rows")
+    return order, rank_of_row, rank_cost
+
+
+def pp_debug_expire_wait(plan: Plan, site: int):
+    """Test hook: lets one bounded wait run out on the plan's status word (see pp_attn.h)."""
+    with torch.cuda.device(plan.workspace.device):
+        _check(lib().pp_debug_expire_wait(plan.handle, int(site), _stream()), "pp_debug_expire_wait")

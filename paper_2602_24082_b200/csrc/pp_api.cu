@@ -8,9 +8,28 @@
 #include <mutex>
 #include <vector>
 
-#include "pp_internal.h"
+#include "pp_dev.cuh"
 
 namespace {
+
+// Test hook: one thread waits on an mbarrier that nobody ever arrives at, with a poll limit of
+// a few thousand instead of the kernels' two million.  No copy and no MMA is in flight, so the
+// give-up path of the bounded wait -- status word, site id, abort flag, return -- can be
+// exercised on a GPU without hanging or faulting anything.
+__global__ void expire_wait_kernel(int32_t* header, int site) {
+  __shared__ __align__(8) unsigned long long bar_storage;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    const uint32_t bar = pp::smem_u32(&bar_storage);
+    pp::mbar_init(bar, 1);
+    abort_flag = 0;
+    pp::fence_mbar_init();
+    const bool done = pp::wait_bar(bar, 0, &abort_flag, header, site, 4096);
+    // a second wait after the give-up returns at once
+    const bool again = pp::wait_bar(bar, 0, &abort_flag, header, site + 1, 4096);
+    if (done || again || !abort_flag) header[1] = -1;
+  }
+}
 
 thread_local int g_last_launches = 0;
 
@@ -109,6 +128,8 @@ int pp_build_plan(const pp_problem* problem, void* d_workspace, size_t workspace
     rc = check_host_descriptors(problem);
     if (rc) return rc;
   }
+  // first call that touches a device: everything above is host-side validation
+  if (!pp::device_is_sm100()) return PP_ERR_UNSUPPORTED;
   pp_plan* plan = new (std::nothrow) pp_plan;
   if (!plan) return PP_ERR_CUDA;
   plan->prob = *problem;
@@ -154,6 +175,20 @@ int pp_build_plan(const pp_problem* problem, void* d_workspace, size_t workspace
     plan->prob.grp_prompt_len = d + n[0];
     plan->prob.grp_resp_off = d + n[0] + n[1];
     plan->prob.resp_len = d + n[0] + n[1] + n[2];
+  } else {
+    // Device descriptors: the first plan kernel copies them into the same block of the
+    // workspace, and the plan (plan kernels, position ids, rotary embedding, loss) reads the
+    // copy -- the caller's arrays are only needed until that kernel has run.
+    int32_t* d = reinterpret_cast<int32_t*>(plan->ws + lay.desc);
+    const size_t n0 = size_t(problem->num_rows) + 1, n1 = size_t(problem->num_groups);
+    plan->src_desc[0] = problem->row_group_off;
+    plan->src_desc[1] = problem->grp_prompt_len;
+    plan->src_desc[2] = problem->grp_resp_off;
+    plan->src_desc[3] = problem->resp_len;
+    plan->prob.row_group_off = d;
+    plan->prob.grp_prompt_len = d + n0;
+    plan->prob.grp_resp_off = d + n0 + n1;
+    plan->prob.resp_len = d + n0 + n1 + n1 + 1;
   }
   if (pp::launch_plan(plan, s, &g_last_launches) != cudaSuccess) {
     delete plan;
@@ -323,7 +358,15 @@ int pp_attn_bwd_noalloc(const pp_plan* plan, const void* q, const void* k, const
     if (!aligned16(p)) return PP_ERR_ALIGNMENT;
   cudaError_t e = pp::launch_bwd_static(plan, q, k, v, o, lse, d_o, softmax_scale, d_q, d_k, d_v,
                                         reinterpret_cast<cudaStream_t>(stream), &g_last_launches);
+  if (e == cudaErrorInvalidDevice) return PP_ERR_INVALID_ARG;  // the plan's device is not current
   return e == cudaSuccess ? PP_OK : (e == cudaErrorNotSupported ? PP_ERR_UNSUPPORTED : PP_ERR_CUDA);
+}
+
+int pp_debug_expire_wait(const pp_plan* plan, int32_t site, pp_stream_t stream) {
+  if (!plan || site < 1) return PP_ERR_INVALID_ARG;
+  expire_wait_kernel<<<1, 32, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+      reinterpret_cast<int32_t*>(plan->ws + plan->lay.header), site);
+  return cudaGetLastError() == cudaSuccess ? PP_OK : PP_ERR_CUDA;
 }
 
 int pp_position_ids(const pp_plan* plan, int32_t* position_ids, pp_stream_t stream) {
@@ -539,13 +582,13 @@ int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_
   auto ok = [](cudaError_t e) { return e == cudaSuccess; };
   if (!ok(cudaEventRecord(ss->e_start, s)) || !ok(cudaStreamWaitEvent(ss->up, ss->e_start, 0)) ||
       !ok(cudaStreamWaitEvent(ss->down, ss->e_start, 0)))
-    return PP_ERR_CUDA;
+    return PP_ERR_CUDA;  // nothing has been given to the side streams yet
   int launches = 0;
   const char* hq = static_cast<const char*>(h_q);
   const char* hk = static_cast<const char*>(h_k);
   const char* hv = static_cast<const char*>(h_v);
   const char* hdo = static_cast<const char*>(h_do);
-  for (size_t c = 0; c < chunks.size(); ++c) {      // all uploads, in order, on the `up` stream
+  for (size_t c = 0; c < chunks.size() && rc == PP_OK; ++c) {  // all uploads, in order, on `up`
     const StepChunk& ch = chunks[c];
     const size_t tc = ch.prob.total_tokens;
     const size_t qo = ch.t0 * Hq * D * 2, ko = ch.t0 * Hkv * D * 2;
@@ -556,7 +599,7 @@ int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_
         !ok(cudaEventRecord(ss->e_qkv[c], ss->up)) ||
         !ok(cudaMemcpyAsync(base + a.d_o + qo, hdo + qo, qb, cudaMemcpyHostToDevice, ss->up)) ||
         !ok(cudaEventRecord(ss->e_do[c], ss->up)))
-      return PP_ERR_CUDA;
+      rc = PP_ERR_CUDA;  // fall through to the join below: copies may already be in flight
   }
   for (size_t c = 0; c < chunks.size() && rc == PP_OK; ++c) {
     const StepChunk& ch = chunks[c];
@@ -646,6 +689,19 @@ int pp_build_rows(int32_t num_groups, int32_t num_responses, const int32_t* grp_
       order, row_group_off, num_rows, reinterpret_cast<long long*>(row_tokens),
       reinterpret_cast<long long*>(row_cost), out_prompt_len, out_resp_off, out_resp_len, status,
       reinterpret_cast<cudaStream_t>(stream), &g_last_launches);
+  return e == cudaSuccess ? PP_OK : PP_ERR_CUDA;
+}
+
+int pp_assign_rows(int32_t num_rows, const int64_t* row_cost, int32_t num_ranks, int32_t* order,
+                   int32_t* rank_of_row, int64_t* rank_cost, pp_stream_t stream) {
+  g_last_launches = 0;
+  if (num_rows < 1 || num_ranks < 1 || !row_cost || !order || !rank_of_row || !rank_cost)
+    return PP_ERR_INVALID_ARG;
+  if (num_rows > 65536 || num_ranks > 1024) return PP_ERR_UNSUPPORTED;
+  cudaError_t e = pp::launch_assign_rows(
+      num_rows, reinterpret_cast<const long long*>(row_cost), num_ranks, order, rank_of_row,
+      reinterpret_cast<long long*>(rank_cost), reinterpret_cast<cudaStream_t>(stream),
+      &g_last_launches);
   return e == cudaSuccess ? PP_OK : PP_ERR_CUDA;
 }
 

@@ -763,6 +763,7 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
   static DeviceSetup setup[kMaxDevices];
   DeviceSetup* dev = device_setup(setup);
   if (!dev) return cudaErrorInvalidDevice;
+  if (dev->cc_major != 10) return cudaErrorNotSupported;
   auto kern = prm.dq_sem ? bwd_kernel<D, true> : bwd_kernel<D, false>;
   if (!dev->configured) {
     cudaError_t e = cudaFuncSetAttribute(bwd_kernel<D, false>,
@@ -777,9 +778,10 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
   const pp_problem& pb = plan->prob;
   const size_t T = pb.total_tokens, Hq = pb.num_q_heads;
   const long long pairs = (long long)T * Hq;
+  const int num_sms = dev->num_sms;
   constexpr int kRowsPerBlock = 8 * (32 / (D / 8)) * 4;  // warps x rows per warp x unroll
-  const unsigned pre_blocks =
-      unsigned(std::min<long long>((pairs + kRowsPerBlock - 1) / kRowsPerBlock, 148 * 16));
+  const unsigned pre_blocks = unsigned(
+      std::min<long long>((pairs + kRowsPerBlock - 1) / kRowsPerBlock, (long long)num_sms * 16));
   auto pre = [&](auto clear, auto token_major) {
     bwd_preprocess_kernel<D, decltype(clear)::value, decltype(token_major)::value>
         <<<pre_blocks, 256, 0, stream>>>(
@@ -794,7 +796,6 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
     if (token_major) pre(std::true_type{}, std::true_type{});
     else pre(std::true_type{}, std::false_type{});
   }
-  const int num_sms = dev->num_sms;
   const long long units = (long long)plan->max_tiles * pb.num_kv_heads;
   dim3 grid(unsigned(std::min<long long>(units, num_sms)));
   ProfileEvents& ev = profile_events();
@@ -805,7 +806,7 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
     ev.bwd_valid = true;
   }
   const size_t n4 = T * Hq * D / 4;
-  unsigned fb = unsigned(std::min<size_t>((n4 + 255) / 256, 148 * 16));
+  unsigned fb = unsigned(std::min<size_t>((n4 + 255) / 256, size_t(num_sms) * 16));
   bwd_finalize_kernel<<<fb, 256, 0, stream>>>(reinterpret_cast<const float4*>(prm.dq_acc),
                                               static_cast<uint2*>(dq), n4, prm.scale);
   if (launches) *launches += 3;
@@ -867,13 +868,20 @@ static __device__ __align__(256) unsigned char g_static_bwd_scratch[kStaticScrat
 
 // In host code `g_static_bwd_scratch` is only a stand-in for the symbol, not a device
 // address, so the address is looked up once per device (with that device current) and kept.
-static cudaError_t static_scratch_address(void** out) {
+// The array used must be the one on the device that holds the plan (and so the tensors): the
+// current device has to be that device, otherwise the call is refused instead of handing the
+// kernels another GPU's array.
+static cudaError_t static_scratch_address(const pp_plan* plan, void** out) {
   static std::mutex mu;
   static void* ptrs[kMaxDevices] = {};
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  cudaPointerAttributes attr;
+  e = cudaPointerGetAttributes(&attr, plan->ws);
+  if (e != cudaSuccess) return e;
+  if (attr.type != cudaMemoryTypeDevice || attr.device != dev) return cudaErrorInvalidDevice;
   std::lock_guard<std::mutex> lock(mu);
   if (!ptrs[dev]) {
     void* p = nullptr;
@@ -890,7 +898,7 @@ cudaError_t launch_bwd_static(const pp_plan* plan, const void* q, const void* k,
                               const void* o, const float* lse, const void* d_o, float scale,
                               void* dq, void* dk, void* dv, cudaStream_t stream, int* launches) {
   void* scratch = nullptr;
-  cudaError_t e = static_scratch_address(&scratch);
+  cudaError_t e = static_scratch_address(plan, &scratch);
   if (e != cudaSuccess) return e;
   // launch_bwd zeroes the fp32 dQ accumulator inside the scratch on every call and rewrites
   // Delta and the scaled LSE, so nothing of an earlier call's contents is read.

@@ -24,7 +24,7 @@ static __device__ unsigned long long g_cta_cycles[256];  // per-CTA busy cycles
 #endif
 
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                         int32_t* header, int site) {
+                                         int32_t* header, int site, uint32_t limit = kSpinLimit) {
 #ifndef PP_TIMING
   if (mbar_try_wait(bar, parity)) return true;  // fast path: already complete
 #endif
@@ -32,7 +32,7 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
 #ifdef PP_TIMING
   const long long t0 = clock64();
 #endif
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+  for (uint32_t it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) {
 #ifdef PP_TIMING
       if (blockIdx.x == 0 && (threadIdx.x & 31) == 0)

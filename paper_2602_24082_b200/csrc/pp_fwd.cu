@@ -618,6 +618,7 @@ cudaError_t launch_fwd_t(const pp_plan* plan, const CUtensorMap& tq, const CUten
   static DeviceSetup setup[kMaxDevices];
   DeviceSetup* dev = device_setup(setup);
   if (!dev) return cudaErrorInvalidDevice;
+  if (dev->cc_major != 10) return cudaErrorNotSupported;
   auto kern = fwd_kernel<D>;
   if (!dev->configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,

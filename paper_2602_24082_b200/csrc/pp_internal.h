@@ -77,7 +77,10 @@ struct PlanLayout {
 }  // namespace pp
 
 struct pp_plan {
-  pp_problem prob;  // descriptor pointers are rewritten to the device copies
+  pp_problem prob;  // descriptor pointers are rewritten to the copies in the workspace
+  // Descriptors given on the device: the caller's arrays, which the first plan kernel copies
+  // into the workspace (null when the host path has staged them already).
+  const int32_t* src_desc[4] = {nullptr, nullptr, nullptr, nullptr};
   int nseg;
   int max_tiles;
   char* ws;
@@ -172,6 +175,7 @@ constexpr int kMaxDevices = 64;
 struct DeviceSetup {
   bool configured = false;
   int num_sms = 0;
+  int cc_major = 0;
 };
 // Entry for the current device in `table` (kMaxDevices entries), or null.
 inline DeviceSetup* device_setup(DeviceSetup* table) {
@@ -179,9 +183,17 @@ inline DeviceSetup* device_setup(DeviceSetup* table) {
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
   DeviceSetup* d = table + dev;
   if (!d->num_sms &&
-      cudaDeviceGetAttribute(&d->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      (cudaDeviceGetAttribute(&d->cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+       cudaDeviceGetAttribute(&d->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess))
     return nullptr;
   return d;
+}
+// The kernels are sm_100a code (tcgen05, tensor memory): any other device is refused before a
+// launch is attempted.  Checked once per device.
+inline bool device_is_sm100() {
+  static DeviceSetup probe[kMaxDevices];
+  DeviceSetup* d = device_setup(probe);
+  return d && d->cc_major == 10;
 }
 
 // Optional event pairs around the forward kernel and the backward main kernel.
@@ -221,6 +233,10 @@ cudaError_t launch_build_rows(int G, int N, const int32_t* prompt_len, const int
                               long long* row_cost, int32_t* out_prompt_len, int32_t* out_resp_off,
                               int32_t* out_resp_len, int32_t* status, cudaStream_t stream,
                               int* launches);
+
+cudaError_t launch_assign_rows(int R, const long long* row_cost, int ranks, int32_t* order,
+                               int32_t* rank_of_row, long long* rank_cost, cudaStream_t stream,
+                               int* launches);
 
 // Size of the scratch array built into the library image for pp_attn_bwd_noalloc.
 constexpr size_t kStaticScratchBytes = size_t(32) << 20;

@@ -16,6 +16,10 @@ namespace {
 
 struct PlanPtrs {
   int32_t* header;
+  // descriptors given on the device: the caller's arrays (null otherwise) and the workspace
+  // block they are copied into, which is what row_group_off .. resp_len below point at
+  const int32_t* src_desc[4];
+  int32_t* desc_copy;
   const int32_t* row_group_off;
   const int32_t* grp_prompt_len;
   const int32_t* grp_resp_off;
@@ -51,6 +55,18 @@ __device__ __forceinline__ bool plan_scan_body(const PlanPtrs& p) {
   __shared__ int32_t s_carry[2];
   const int tid = threadIdx.x;
 
+  // Descriptors handed over on the device are copied into the workspace first: everything
+  // after this call -- the later plan kernels, position ids, rotary embedding, the loss -- reads
+  // the copy, so the caller's arrays are free again once this kernel has run.
+  if (p.src_desc[0]) {
+    const int n[4] = {p.num_rows + 1, p.G, p.G + 1, p.N};
+    int32_t* dst = p.desc_copy;
+    for (int a = 0; a < 4; ++a) {
+      for (int i = tid; i < n[a]; i += blockDim.x) dst[i] = p.src_desc[a][i];
+      dst += n[a];
+    }
+    __syncthreads();
+  }
   if (tid == 0) {
     p.header[0] = kStatusOk;
     p.header[1] = 0;
@@ -494,6 +510,8 @@ cudaError_t launch_plan(const pp_plan* plan, cudaStream_t stream, int* launches)
   char* ws = plan->ws;
   const PlanLayout& l = plan->lay;
   p.header = reinterpret_cast<int32_t*>(ws + l.header);
+  for (int a = 0; a < 4; ++a) p.src_desc[a] = plan->src_desc[a];
+  p.desc_copy = reinterpret_cast<int32_t*>(ws + l.desc);
   p.row_group_off = plan->prob.row_group_off;
   p.grp_prompt_len = plan->prob.grp_prompt_len;
   p.grp_resp_off = plan->prob.grp_resp_off;

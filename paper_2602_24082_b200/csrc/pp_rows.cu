@@ -1,8 +1,8 @@
-// Row builder: the step before the attention path (paper Sec. 2.3, used in Sec. 4.3).
-// Preference groups [prompt | responses] of varying length are ordered by total length,
-// longest first with ties in their original order ("batch sorting": samples of similar length
-// end up together), and consecutive groups of that order are concatenated into rows of at most
-// `capacity` tokens ("packing ... up to a maximum sequence length": next fit).  The outputs are
+// Row builder: the step before the attention path (paper Sec. 2.2, used with preference
+// packing in Sec. 5.2).  Preference groups [prompt | responses] of varying length are ordered by
+// total length, longest first with ties in their original order (batch sorting: samples of
+// similar length end up together), and consecutive groups of that order are concatenated into
+// rows of at most `capacity` tokens (batch packing: next fit).  The outputs are
 // the order, the rows, each row's tokens and visible query-key pairs (the attention cost of
 // Sec. 3.2.1, for balancing data-parallel ranks) and the descriptor arrays in row order, ready
 // for pp_build_plan with descriptors on the device.  Integer work only; microseconds.
@@ -208,7 +208,80 @@ __global__ void __launch_bounds__(1024) rows_pack_kernel(RowsPtrs p) {
   }
 }
 
+// ---------------------------------------------------------------- rows -> data-parallel ranks
+// Longest-processing-time assignment: rows in order of decreasing cost (ties by index), each to
+// the rank with the least cost so far (ties to the lowest rank).  The order comes from rank
+// counting over all rows; the greedy pass is sequential by nature and runs in one warp, the
+// lanes sharing the search for the least-loaded rank.
+__global__ void __launch_bounds__(256)
+assign_rank_kernel(int R, const long long* __restrict__ cost, int32_t* __restrict__ order) {
+  __shared__ long long s_c[256];
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  const long long mine = r < R ? cost[r] : 0;
+  int rank = 0;
+  for (int base = 0; base < R; base += 256) {
+    const int u = base + threadIdx.x;
+    s_c[threadIdx.x] = u < R ? cost[u] : -1;
+    __syncthreads();
+    const int lim = min(256, R - base);
+    for (int i = 0; i < lim; ++i) {
+      const long long o = s_c[i];
+      rank += (o > mine) || (o == mine && base + i < r);
+    }
+    __syncthreads();
+  }
+  if (r < R) order[rank] = r;
+}
+
+constexpr int kMaxAssignRanks = 1024;
+
+__global__ void __launch_bounds__(32)
+assign_greedy_kernel(int R, int ranks, const long long* __restrict__ cost,
+                     const int32_t* __restrict__ order, int32_t* __restrict__ rank_of_row,
+                     long long* __restrict__ rank_cost) {
+  __shared__ long long s_load[kMaxAssignRanks];
+  const int lane = threadIdx.x;
+  for (int k = lane; k < ranks; k += 32) s_load[k] = 0;
+  __syncwarp();
+  for (int i = 0; i < R; ++i) {
+    long long best = 0x7fffffffffffffffLL;
+    int best_k = ranks;
+    for (int k = lane; k < ranks; k += 32) {   // ascending k: the first minimum is kept
+      const long long l = s_load[k];
+      if (l < best) {
+        best = l;
+        best_k = k;
+      }
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      const long long ob = __shfl_xor_sync(0xffffffffu, best, d);
+      const int ok = __shfl_xor_sync(0xffffffffu, best_k, d);
+      if (ob < best || (ob == best && ok < best_k)) {
+        best = ob;
+        best_k = ok;
+      }
+    }
+    if (lane == 0) {
+      const int row = order[i];
+      rank_of_row[row] = best_k;
+      s_load[best_k] = best + cost[row];
+    }
+    __syncwarp();
+  }
+  for (int k = lane; k < ranks; k += 32) rank_cost[k] = s_load[k];
+}
+
 }  // namespace
+
+cudaError_t launch_assign_rows(int R, const long long* row_cost, int ranks, int32_t* order,
+                               int32_t* rank_of_row, long long* rank_cost, cudaStream_t stream,
+                               int* launches) {
+  assign_rank_kernel<<<(R + 255) / 256, 256, 0, stream>>>(R, row_cost, order);
+  assign_greedy_kernel<<<1, 32, 0, stream>>>(R, ranks, row_cost, order, rank_of_row, rank_cost);
+  if (launches) *launches = 2;
+  return cudaGetLastError();
+}
 
 size_t rows_workspace_bytes(int G) {
   return align_up(size_t(8) * G, 256) * 3 + align_up(size_t(4) * G, 256) * 4;

@@ -7,7 +7,8 @@ own: a MAX over ranks of the timed region and a SUM of the work done.
 """
 from __future__ import annotations
 
-from typing import Tuple
+import dataclasses
+from typing import List, Sequence, Tuple
 
 import torch
 import torch.distributed as dist
@@ -36,3 +37,30 @@ def whole_job_throughput(total_ms: float, steps: int, flops_per_step_all_ranks: 
     """Useful TFLOP/s of the whole job: all ranks' FLOPs per step over the slowest rank's
     time per step."""
     return flops_per_step_all_ranks / (total_ms / steps * 1e-3) / 1e12
+
+
+def pool_rows(batches: Sequence) -> Tuple[List[Tuple[int, int]], List[int]]:
+    """All rows of the ranks' batches as (batch, row) pairs, with each row's attention cost
+    (visible query-key pairs, paper Sec. 3.2.1) -- the input of the row assignment."""
+    pool = [(b, r) for b, w in enumerate(batches) for r in range(len(w.rows))]
+    costs = [int(batches[b].select_rows([r]).useful_pairs()) for (b, r) in pool]
+    return pool, costs
+
+
+def rank_batch(batches: Sequence, pool: Sequence[Tuple[int, int]], rank_of_row: Sequence[int], rank: int):
+    """The workload of one rank: the pooled rows assigned to it, in pool order (paper Sec. 2.2:
+    rows are dealt out so that no rank waits for the one with the longest sequences).  A rank
+    that got no row keeps the shortest row of the pool, so that every rank has work to time."""
+    mine = [i for i, k in enumerate(rank_of_row) if k == rank]
+    if not mine:
+        mine = [min(range(len(pool)), key=lambda i: batches[pool[i][0]].row_lengths()[pool[i][1]])]
+    rows, lv, off = [], [], 0
+    for i in mine:
+        b, r = pool[i]
+        sub = batches[b].select_rows([r])
+        rows.extend(sub.rows)
+        lv.extend((lo + off, hi + off) for (lo, hi) in sub.low_var_ranges)
+        off += sub.total_tokens
+    t = batches[0]
+    return dataclasses.replace(t, name=f"{t.name}/rank{rank}", rows=rows, low_var_ranges=lv,
+                               seed=t.seed + 1000 * rank)

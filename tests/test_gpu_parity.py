@@ -167,7 +167,7 @@ def _subset_parity(w, row_ids, kv_heads):
     check_against_oracle(sub, stens, cut)
 
 
-def _group_parity(w, groups, kv_heads):
+def _group_parity(w, groups, kv_heads, deterministic=False):
     """Run the GPU on the whole workload at full size (the launch configuration the benchmark
     times), then check whole groups x KV-head groups -- independent units -- element by
     element against the oracle."""
@@ -177,7 +177,8 @@ def _group_parity(w, groups, kv_heads):
     plan = B.plan_for(w, desc_on_device=True)
     plan.bwd_scratch().fill_(0xFF)
     o, lse = B.pp_attn_fwd(plan, q, k, v, w.softmax_scale, for_backward=True)
-    dq, dk, dv = B.pp_attn_bwd(plan, q, k, v, o, lse, do, w.softmax_scale)
+    dq, dk, dv = B.pp_attn_bwd(plan, q, k, v, o, lse, do, w.softmax_scale,
+                               deterministic=deterministic)
     torch.cuda.synchronize()
     assert plan.status() == (0, 0)
     sub, stens, tok, qh = W.slice_groups(w, tens, groups, kv_heads)
@@ -233,6 +234,36 @@ def test_config3_full_size_sampled_groups():
 def test_config4_full_size_sampled_group(point):
     w = W.config4(point)
     _group_parity(w, _smallest_groups(w, 1), [point % 8])
+
+
+def _largest_groups(w, n):
+    sizes = sorted(((p + sum(rs), ri, gi) for ri, row in enumerate(w.rows) for gi, (p, rs) in enumerate(row)),
+                   reverse=True)
+    return [(ri, gi) for (_, ri, gi) in sizes[:n]]
+
+
+# The long end of every full-size configuration: forward units of more than a hundred key
+# tiles, backward units that walk every query tile of a 16K-token group for all query heads of
+# the KV head.  One whole group x one KV-head group each (independent of everything else in
+# the launch), element by element against the oracle.
+def test_config2_full_size_largest_row():
+    w = W.config2()
+    _group_parity(w, _largest_groups(w, 1), [1])
+
+
+def test_config3_full_size_largest_group():
+    w = W.config3()
+    _group_parity(w, _largest_groups(w, 1), [3])
+
+
+@pytest.mark.parametrize("point,det", [(2, False), (5, False), (0, True)],
+                         ids=["rho4-n2", "rho16-n4", "rho1-n2-deterministic"])
+def test_config4_full_size_largest_group(point, det):
+    w = W.config4(point)
+    big = _largest_groups(w, 1)
+    p, rs = w.rows[big[0][0]][big[0][1]]
+    assert p + sum(rs) >= 12000
+    _group_parity(w, big, [(point + 3) % 8], deterministic=det)
 
 
 def test_many_tiny_groups_multi_kernel_plan():

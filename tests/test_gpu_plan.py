@@ -204,3 +204,71 @@ def test_host_descriptors_reach_the_device_unchanged(groups):
     assert np.array_equal(t0, t1) and np.array_equal(f0, f1) and np.array_equal(k0, k1)
     assert np.array_equal(b0[:nb], b1[:nb])      # entries past the backward tiles are unused
     assert np.array_equal(got.read_bwd_units(nb), want.read_bwd_units(nb))
+
+
+def test_bounded_wait_gives_up_and_later_kernels_do_nothing():
+    """A wait that runs out (one thread, no copy or MMA in flight, 4096 polls on a barrier that
+    nobody arrives at) records status 3 with its site id and returns; the kernels of later
+    calls on that plan then return at once and leave the outputs untouched."""
+    from paper_2602_24082_b200 import binding as B
+    w = W.Workload("expire", [[(150, (70, 33))]], 2, 1, 64, seed=3)
+    q, k, v, do = (x.cuda() for x in w.tensors())
+    plan = B.plan_for(w)
+    o, lse = B.pp_attn_fwd(plan, q, k, v, w.softmax_scale)
+    torch.cuda.synchronize()
+    assert plan.status() == (0, 0)
+    B.pp_debug_expire_wait(plan, 57)
+    torch.cuda.synchronize()
+    assert plan.status() == (3, 57)
+    o2 = torch.full_like(q, 7.0)
+    dq, dk, dv = torch.full_like(q, 7.0), torch.full_like(k, 7.0), torch.full_like(v, 7.0)
+    B.pp_attn_fwd(plan, q, k, v, w.softmax_scale, o=o2)
+    B.pp_attn_bwd(plan, q, k, v, o, lse, do, w.softmax_scale, d_q=dq, d_k=dk, d_v=dv)
+    torch.cuda.synchronize()
+    assert plan.status() == (3, 57)
+    assert (o2 == 7.0).all() and (dk == 7.0).all() and (dv == 7.0).all()
+    # a fresh plan in the same workspace works again
+    plan2 = B.pp_build_plan(w.descriptors(), 2, 1, 64, w.total_tokens, workspace=plan.workspace)
+    o3, _ = B.pp_attn_fwd(plan2, q, k, v, w.softmax_scale)
+    torch.cuda.synchronize()
+    assert plan2.status() == (0, 0) and torch.equal(o3, o)
+
+
+def test_device_descriptors_are_copied_by_the_plan():
+    """Descriptors given on the device are only read by the first plan kernel: overwriting the
+    caller's arrays afterwards changes nothing for the plan's later users (position ids,
+    rotary embedding, loss)."""
+    from oracle import loss as OL
+    from oracle import rope as OR
+    from paper_2602_24082_b200 import binding as B
+    w = W.Workload("desc-copy", [[(97, (64, 200)), (128, (128, 31))], [(5, (3, 1, 9))]], 2, 1, 64, seed=8)
+    desc = w.descriptors()
+    desc_dev = [torch.from_numpy(np.ascontiguousarray(a)).cuda() for a in desc]
+    plan = B.pp_build_plan(desc, 2, 1, 64, w.total_tokens, device_arrays=desc_dev)
+    torch.cuda.synchronize()
+    for t in desc_dev:
+        t.fill_(-12345)
+    torch.cuda.synchronize()
+    pos = B.pp_position_ids(plan).cpu().numpy()
+    assert np.array_equal(pos.astype(np.int64), OR.position_ids(w.rows))
+    rng = np.random.default_rng(2)
+    lp = (-rng.gamma(2.0, 1.0, w.total_tokens)).astype(np.float32)
+    s, r, loss, grad = B.pp_preference_loss(plan, torch.from_numpy(lp).cuda(), None, 0.05)
+    S, Rw, Ls, G = OL.preference_loss(w.rows, lp, None, 0.05)
+    assert np.abs(s.cpu().numpy() - S).max() <= 1e-4 * max(1.0, np.abs(S).max())
+    assert np.abs(loss.cpu().numpy() - Ls).max() <= 1e-4 * max(1.0, np.abs(Ls).max())
+    q, k, _, _ = w.tensors()
+    qd, kd = q.cuda().clone(), k.cuda().clone()
+    B.pp_rope_qk(plan, qd, kd, 10000.0)
+    ref = OR.rope(q.double().numpy(), OR.position_ids(w.rows), 10000.0)
+    assert np.abs(qd.float().cpu().numpy() - ref).max() <= 2e-2
+    assert plan.status() == (0, 0)
+
+
+def test_this_device_passes_the_compute_capability_check():
+    """pp_build_plan refuses devices that are not compute capability 10.x with
+    PP_ERR_UNSUPPORTED; the B200 the suite runs on must pass."""
+    from paper_2602_24082_b200 import binding as B
+    assert torch.cuda.get_device_capability(0)[0] == 10
+    plan = B.plan_for(W.config0())
+    assert plan.status() == (0, 0)

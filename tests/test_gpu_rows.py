@@ -82,3 +82,44 @@ def test_output_feeds_the_plan_builder():
     assert plan.status() == (0, 0)
     tiles = plan.read()[0]
     assert int(tiles[:, 1].sum()) == T
+
+
+@pytest.mark.parametrize("rows,ranks,seed", [(1, 1, 0), (6, 3, 1), (3, 8, 2), (100, 8, 3), (777, 64, 4),
+                                             (5000, 1024, 5), (4096, 7, 6)])
+def test_assign_rows_matches_the_oracle_bit_for_bit(rows, ranks, seed):
+    from paper_2602_24082_b200 import binding as B
+    rng = np.random.default_rng(seed)
+    cost = rng.integers(0, 1 << 40, size=rows).astype(np.int64)
+    if seed == 3:
+        cost[::3] = cost[0]                      # ties
+    order, rank_of_row, rank_cost = B.pp_assign_rows(torch.from_numpy(cost).cuda(), ranks)
+    want = R.assign_rows(cost, ranks)
+    assert np.array_equal(order.cpu().numpy(), want[0])
+    assert np.array_equal(rank_of_row.cpu().numpy(), want[1])
+    assert np.array_equal(rank_cost.cpu().numpy(), want[2])
+
+
+def test_assign_rows_worked_example_and_hand_over_from_the_row_builder():
+    from paper_2602_24082_b200 import binding as B
+    order, rank_of_row, rank_cost = B.pp_assign_rows(torch.tensor([7, 3, 9, 3, 5, 1], dtype=torch.int64).cuda(), 3)
+    assert rank_of_row.tolist() == [1, 2, 0, 1, 2, 2] and rank_cost.tolist() == [9, 10, 9]
+    rng = np.random.default_rng(9)
+    P, off, rl = _random_groups(rng, 400, 500)
+    tok = R.group_tokens(P, off, rl)
+    got = _gpu(P, off, rl, int(tok.max() * 3))
+    o2, r2, c2 = B.pp_assign_rows(got["row_cost"], 8)           # device to device, no copy back
+    want = R.assign_rows(got["row_cost"].cpu().numpy(), 8)
+    assert np.array_equal(r2.cpu().numpy(), want[1]) and np.array_equal(c2.cpu().numpy(), want[2])
+    cost = got["row_cost"].cpu().numpy()
+    assert c2.max().item() <= cost.sum() / 8 + cost.max()
+
+
+def test_assign_rows_errors():
+    from paper_2602_24082_b200 import binding as B
+    c = torch.ones(4, dtype=torch.int64).cuda()
+    with pytest.raises(B.PPError) as e:
+        B.pp_assign_rows(c, 0)
+    assert e.value.code == -1
+    with pytest.raises(B.PPError) as e:
+        B.pp_assign_rows(c, 2000)
+    assert e.value.code == -2

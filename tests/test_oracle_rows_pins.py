@@ -89,3 +89,57 @@ def test_pair_count_matches_dense_mask():
         m = oracle.dense_mask(desc, 0)
         assert int(m.sum()) == int(want[g])
     assert int(R.group_tokens(P, off, rl).sum()) == int(P.sum() + rl.sum())
+
+
+# ---------------------------------------------------------------- rows -> ranks
+ASSIGN_GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "assign_example.txt")
+
+
+def test_assign_worked_example():
+    kv = {}
+    for line in open(ASSIGN_GOLDEN):
+        if line.startswith("#") or not line.strip():
+            continue
+        k, *v = line.split()
+        kv[k] = [int(x) for x in v]
+    order, rank_of_row, rank_cost = R.assign_rows(kv["row_cost"], kv["ranks"][0])
+    assert order.tolist() == kv["order"]
+    assert rank_of_row.tolist() == kv["rank_of_row"]
+    assert rank_cost.tolist() == kv["rank_cost"]
+
+
+def _best_makespan(cost, m):
+    """Brute force over all m^n assignments (tiny n only)."""
+    import itertools
+    best = None
+    for assign in itertools.product(range(m), repeat=len(cost)):
+        load = [0] * m
+        for c, k in zip(cost, assign):
+            load[k] += c
+        best = max(load) if best is None else min(best, max(load))
+    return best
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_assign_properties_and_bound_against_brute_force(seed):
+    rng = np.random.default_rng(100 + seed)
+    n, m = int(rng.integers(1, 9)), int(rng.integers(1, 4))
+    cost = rng.integers(0, 50, size=n).tolist()
+    order, rank_of_row, rank_cost = R.assign_rows(cost, m)
+    assert sorted(order.tolist()) == list(range(n))                       # a permutation
+    assert all(cost[order[i]] >= cost[order[i + 1]] for i in range(n - 1))  # decreasing cost
+    load = [sum(c for c, k in zip(cost, rank_of_row) if k == r) for r in range(m)]
+    assert load == rank_cost.tolist() and sum(load) == sum(cost)
+    # list scheduling: the fullest rank got its last row while it was the emptiest
+    assert max(load) <= sum(cost) / m + max(cost)
+    # longest-processing-time rule: within (4/3 - 1/(3m)) of the optimum (Graham 1969)
+    opt = _best_makespan(cost, m)
+    assert max(load) <= (4.0 / 3.0 - 1.0 / (3 * m)) * opt + 1e-9
+
+
+def test_assign_ties_and_more_ranks_than_rows():
+    order, rank_of_row, rank_cost = R.assign_rows([5, 5, 5], 5)
+    assert order.tolist() == [0, 1, 2] and rank_of_row.tolist() == [0, 1, 2]
+    assert rank_cost.tolist() == [5, 5, 5, 0, 0]
+    order, rank_of_row, rank_cost = R.assign_rows([0, 0, 7], 2)
+    assert order.tolist() == [2, 0, 1] and rank_of_row.tolist() == [1, 1, 0]
