@@ -1,6 +1,7 @@
 """The device-built plan against a host re-derivation from the dense mask."""
 import numpy as np
 import pytest
+import torch
 
 import oracle
 from paper_2602_24082_b200 import workloads as W
