@@ -127,10 +127,11 @@ int pp_destroy_plan(pp_plan* plan);
 int pp_plan_max_tiles(const pp_plan* plan);
 /* The backward's key tiles: each GROUP (prompt and responses as one token range) cut into
  * tiles of 128 tokens from the group's start, so a tile may straddle segments.  Each record is
- * 8 int32: {start, len, vis_end, full_end, grp_start, grp_end, work, npc}: queries
- * [start, vis_end) see at least one key of the tile, queries [start + len, full_end) see all
- * of them, work = number of 128-token query tiles from `start` that reach vis_end, npc =
- * number of tiles of the group that hold prompt keys.
+ * 8 int32: {start, len, vis_end, dep_lo, grp_start, grp_end, work, npc}: queries
+ * [start, vis_end) see at least one key of the tile, work = number of 128-token query tiles
+ * from `start` that reach vis_end, npc = number of tiles of the group that hold prompt keys;
+ * read as a query tile, the key tiles that add to its dQ are the group's tiles [0, npc) and
+ * [dep_lo, own index] (group-relative indices).
  * *num_tiles receives their count (at most pp_plan_max_tiles).  Synchronises `stream`. */
 int pp_plan_read_bwd_tiles(const pp_plan* plan, pp_stream_t stream, int32_t* num_tiles,
                            int32_t* btiles);
@@ -173,9 +174,11 @@ int pp_attn_bwd(const pp_plan* plan, const void* q, const void* k, const void* v
  * Sec. 3.2's equivalence to unpacked training is what a reproducible gradient lets a user
  * verify run against run).  pp_attn_bwd adds the per-key-tile contributions to a query tile's
  * dQ in whatever order the CTAs reach it, so dQ can differ in the last bits between runs; here
- * the key tiles of a group take turns in ascending tile order (one counter per query tile and
- * head inside d_scratch, units handed out in ascending tile order so that no CTA waits for
- * work that has not started).  dK, dV and the forward are reproducible in both variants.
+ * the key tiles of a group take turns in descending tile order -- the order in which the units,
+ * each walking its query tiles upwards from its own tile, reach a query tile anyway -- (one
+ * counter per query tile and head inside d_scratch; units handed out one (group, KV head) set
+ * after the other and in descending tile order inside a set, so that no CTA waits for work
+ * that has not started).  dK, dV and the forward are reproducible in both variants.
  * Same arguments, sizes and errors as pp_attn_bwd; a turn that does not come within a bounded
  * number of polls sets the plan's status word (PP_ERR_PLAN_STATUS from pp_plan_status).
  */

@@ -141,7 +141,7 @@ class Plan:
         return tiles[:n.value], fo[:n.value], bo[:n.value], ke
 
     def read_bwd_tiles(self) -> np.ndarray:
-        """Backward key tiles [n, 8]: start, len, vis_end, full_end, grp_start, grp_end, work, npc."""
+        """Backward key tiles [n, 8]: start, len, vis_end, dep_lo, grp_start, grp_end, work, npc."""
         mt = lib().pp_plan_max_tiles(self.handle)
         bt = np.zeros((mt, 8), dtype=np.int32)
         n = ctypes.c_int32(0)

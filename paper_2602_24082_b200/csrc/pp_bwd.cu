@@ -625,20 +625,41 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     for (; get_bwd_unit(prm, take_unit(ucnt, true), ntiles_total, un); ++ucnt) {
       QIter qi;
       // Deterministic variant: the key tiles that add to a (query tile, head) do so in
-      // ascending tile order.  The counter of the pair holds 1 + the group-relative index of
-      // the last key tile that has added (0: none yet); this unit's turn comes when it shows
-      // the previous contributor -- the tile before this one if that tile reaches the query
-      // tile, else the group's last tile with prompt keys.  In this variant units are handed
-      // out in ascending tile order within a group (the plan's second unit list), so the tile
-      // waited for is always running or done and the waits cannot lock up.
+      // DESCENDING tile order: the query tile's own key tile first, then the tiles below it
+      // down to dep_lo of the query tile, then the prompt tiles from npc - 1 down to 0.  With
+      // every unit walking its query tiles upwards from its own tile, that is the order in
+      // which the units reach a query tile anyway (tile k gets there one query tile's worth
+      // of iterations after tile k + 1), so in the steady state nobody waits.  The counter of
+      // the pair holds 1 + the group-relative index of the last key tile that has added (0:
+      // none yet).  Units are handed out set by set and inside a set in descending tile order
+      // (the plan's second unit list), so the tile waited for is always running or done and
+      // the waits cannot lock up.
       const int k_rel = (un.tile.start - un.tile.grp_start) / kTile;
-      int prev_vis_end = 0;
-      if (kDet && leader && k_rel > 0) prev_vis_end = prm.tiles[un.tidx - 1].vis_end;
+      int dep_lo = 0;
+      // Passing the turn on needs the reductions of the tile to be complete (a wait of a
+      // microsecond or two), so it is deferred: the counter of iteration i is published after
+      // the reductions of iteration i + 1 have been issued -- the next key tile gets to the
+      // same query tile a whole query tile's worth of iterations later -- or at once whenever
+      // this unit finds that it has to wait for its own turn.
+      int32_t* pend = nullptr;
+      auto publish = [&](int32_t* p) {   // (the release store orders it behind the completed adds)
+        const int mine = k_rel + 1;
+        asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(mine) : "memory");
+      };
       for (int it = 0; it < un.n_it; ++it, q_advance(qi, prm.Hq / prm.Hkv)) {
         const QTile qt = q_tile_at(prm, un, qi);
         const uint32_t g = gc + it;
         int32_t* sem = nullptr;
-        if (kDet && leader) sem = prm.dq_sem + size_t(un.tidx + qi.qt) * prm.Hq + qt.h;
+        int seen_early = -1;
+        if (kDet && leader) {
+          sem = prm.dq_sem + size_t(un.tidx + qi.qt) * prm.Hq + qt.h;
+          // the last prompt tile follows the lowest response tile that adds to this query tile
+          if (qi.hh == 0 && qi.qt > 0 && k_rel == un.tile.npc - 1 && k_rel + qi.qt >= un.tile.npc)
+            dep_lo = prm.tiles[un.tidx + qi.qt].dep_lo;
+          // read the counter now: the answer (normally already the expected one) is back by the
+          // time the first box of the tile is staged
+          asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen_early) : "l"(sem) : "memory");
+        }
         wait_bar(bar(kDqFull), g & 1, abort_flag, prm.header, 80);
         tc_fence_after();
         // Two halves of D/2 columns.  The second half is read out of tensor memory (and the
@@ -680,14 +701,21 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             if (leader) {
               if (kDet && sem && half == 0 && c == 0) {  // wait for this unit's turn (bounded)
                 const int expect =
-                    k_rel == 0 ? 0 : (prev_vis_end > qt.start ? k_rel : un.tile.npc);
-                bool ok = false;
-                for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
+                    qi.qt == 0 ? 0
+                               : ((k_rel == un.tile.npc - 1 && k_rel + qi.qt >= un.tile.npc) ? dep_lo + 1
+                                                                                            : k_rel + 2);
+                bool ok = seen_early == expect;
+                for (uint32_t spin = 0; !ok && spin < (1u << 22); ++spin) {
                   int seen;
                   asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(sem) : "memory");
                   if (seen == expect) {
                     ok = true;
                     break;
+                  }
+                  if (pend) {  // about to wait: do not keep the unit below waiting for us
+                    bulk_wait_group<0>();
+                    publish(pend);
+                    pend = nullptr;
                   }
                   if ((spin & 0xff) == 0xff && *abort_flag) break;
                   __nanosleep(20);
@@ -703,12 +731,17 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             }
           }
         }
-        if (kDet && sem) {  // all four boxes of the tile added and visible: pass the turn on
-          bulk_wait_group<0>();
-          __threadfence();
-          const int mine = k_rel + 1;
-          asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(sem), "r"(mine) : "memory");
+        if (kDet && sem) {
+          if (pend) {  // the previous tile's boxes (all but this tile's D / 32 groups) have landed
+            bulk_wait_group<D / 32>();
+            publish(pend);
+          }
+          pend = sem;
         }
+      }
+      if (kDet && pend) {
+        bulk_wait_group<0>();
+        publish(pend);
       }
       gc += un.n_it;
     }

@@ -33,8 +33,8 @@ struct BTile {
   int32_t start;      // first token
   int32_t len;        // 1..128 tokens
   int32_t vis_end;    // largest key_end of the tile's keys: queries [start, vis_end) see some key
-  int32_t full_end;   // smallest key_end of the tile's keys: queries in [start + len, full_end)
-                      //   see every key of the tile
+  int32_t dep_lo;     // read as a query tile: besides the prompt tiles [0, npc), the key tiles
+                      //   [dep_lo, own index] of the group's grid add to its dQ
   int32_t grp_start;  // first token of the group (also the group's identity)
   int32_t grp_end;    // one past the last token of the group
   int32_t work;       // number of query tiles: 1 + ceil((vis_end - start - len) / 128)
@@ -68,8 +68,8 @@ struct PlanLayout {
   size_t tile_gwork; // int32[max_tiles]  backward work of the backward tile's whole group
   size_t tile_sgroup; // int32[max_tiles] super-group (block of consecutive groups)
   size_t bwd_units;  // int32[max_tiles * Hkv]  (kv head << 24) | backward tile, processing order
-  size_t bwd_units_det;  // the same units, inside a super-group by ascending tile index: the
-                         //   order of the deterministic backward
+  size_t bwd_units_det;  // the same units, one (group, KV head) set after the other and inside a
+                         //   set by descending tile index: the order of the deterministic backward
   size_t key_end;    // int32[T]
   size_t total;
 };

@@ -9,6 +9,8 @@
 // backward has its own key tiles, cut per group (see BTile): its masks are two comparisons per
 // element with per-key bounds, so straddling costs nothing there and short segments leave no
 // ragged tiles.
+#include <algorithm>
+
 #include "pp_internal.h"
 
 namespace pp {
@@ -37,6 +39,7 @@ struct PlanPtrs {
   int32_t* bwd_units_det;
   int Hkv;
   int32_t* key_end;
+  int det_asc_max;  // deterministic order: sets of at most this many tiles are handed out longest first
   int num_rows, G, N, T, nseg, max_tiles;
 };
 
@@ -260,10 +263,14 @@ __device__ __forceinline__ void plan_btile_body(const PlanPtrs& p, int t) {
   // key_end is the group's end for prompt keys and the own response's end otherwise; along
   // the tile it is: (group end for the prompt part,) then increasing response ends
   b.vis_end = (s_first == sp) ? ge : p.seg_start[s_last + 1];
-  if (s_last == sp) b.full_end = ge;                              // prompt keys only
-  else b.full_end = p.seg_start[(s_first == sp ? sp + 1 : s_first) + 1];  // first response part
   b.work = 1 + (b.vis_end - (b.start + b.len) + kTile - 1) / kTile;
   b.npc = (pe - gs + kTile - 1) / kTile;
+  // Read as a QUERY tile: the key tiles that add to its dQ are the prompt tiles [0, npc) and
+  // the tiles [dep_lo, own index] -- from the one holding the start of the first row's own
+  // response on (earlier tiles past the prompt hold only earlier responses' keys).
+  const int k_rel = (b.start - gs) / kTile;
+  b.dep_lo = k_rel;
+  if (b.start >= pe) b.dep_lo = max(b.npc, (p.seg_start[s_first] - gs) / kTile);
   p.btiles[t] = b;
 }
 
@@ -334,14 +341,24 @@ __device__ __forceinline__ void plan_units_body(const PlanPtrs& p, int t, int n)
     pos += (osg > sg) || (osg == sg && ((ob > wb) || (ob == wb && u < t)));
   }
   for (int kvh = 0; kvh < p.Hkv; ++kvh) p.bwd_units[p.Hkv * pos + kvh] = (kvh << 24) | t;
-  // deterministic order: inside a super-group by ascending tile index, so that every tile of
-  // a group is handed out after the group's earlier tiles
-  int dpos = 0;
+  // Deterministic order: one (group, KV head) set after the other, groups by decreasing work.
+  // The tiles add to a query tile's dQ in descending order, so a unit waits for the unit of the
+  // next tile.  Inside a set the units go out in ascending tile order (longest first, as in the
+  // default order) when the set is small against the grid: only the one set at the frontier of
+  // the list can have units waiting for a unit that has not been handed out yet, so fewer than
+  // det_asc_max CTAs can be held up that way and the others keep drawing.  Larger sets go out
+  // in DESCENDING tile order, where every unit follows the units it waits for.
+  const int gs = p.btiles[t].grp_start, gw = p.tile_gwork[t];
+  int before = 0, ng = 0;  // tiles of groups ranked earlier; tiles of this group
   for (int u = 0; u < n; ++u) {
-    const int osg = p.tile_sgroup[u];
-    dpos += (osg > sg) || (osg == sg && u < t);
+    const int ogs = p.btiles[u].grp_start, ow = p.tile_gwork[u];
+    before += (ow > gw) || (ow == gw && ogs < gs);
+    ng += (ogs == gs);
   }
-  for (int kvh = 0; kvh < p.Hkv; ++kvh) p.bwd_units_det[p.Hkv * dpos + kvh] = (kvh << 24) | t;
+  const int k_rel = (p.btiles[t].start - gs) / kTile;
+  const int slot = ng <= p.det_asc_max ? k_rel : ng - 1 - k_rel;
+  for (int kvh = 0; kvh < p.Hkv; ++kvh)
+    p.bwd_units_det[p.Hkv * before + kvh * ng + slot] = (kvh << 24) | t;
 }
 
 __global__ void plan_gwork_kernel(PlanPtrs p) {
@@ -450,19 +467,24 @@ __global__ void __launch_bounds__(1024) plan_fused_kernel(PlanPtrs p) {
   }
   __syncthreads();
   for (int t = wid; t < nb; t += nwarp) {
-    const int sg = s_sg[t], wb = s_wb[t];
-    int pos = 0, dpos = 0;
+    const int sg = s_sg[t], wb = s_wb[t], gs = s_gs[t], gw = s_gw[t];
+    int pos = 0, before = 0, ng = 0, k_rel = 0;
     for (int u = lane; u < nb; u += 32) {
-      const int osg = s_sg[u], ob = s_wb[u];
+      const int osg = s_sg[u], ob = s_wb[u], ogs = s_gs[u], ow = s_gw[u];
       pos += (osg > sg) || (osg == sg && ((ob > wb) || (ob == wb && u < t)));
-      dpos += (osg > sg) || (osg == sg && u < t);
+      before += (ow > gw) || (ow == gw && ogs < gs);
+      ng += (ogs == gs);
+      k_rel += (ogs == gs && u < t);   // tiles of a group are consecutive
     }
     pos = warp_sum(pos);
-    dpos = warp_sum(dpos);
-    // ascending tiles inside a super-group for the deterministic backward
+    before = warp_sum(before);
+    ng = warp_sum(ng);
+    k_rel = warp_sum(k_rel);
+    // deterministic backward: set after set (see plan_units_body)
+    const int slot = ng <= p.det_asc_max ? k_rel : ng - 1 - k_rel;
     for (int kvh = lane; kvh < p.Hkv; kvh += 32) {
       p.bwd_units[p.Hkv * pos + kvh] = (kvh << 24) | t;
-      p.bwd_units_det[p.Hkv * dpos + kvh] = (kvh << 24) | t;
+      p.bwd_units_det[p.Hkv * before + kvh * ng + slot] = (kvh << 24) | t;
     }
   }
 }
@@ -529,6 +551,12 @@ cudaError_t launch_plan(const pp_plan* plan, cudaStream_t stream, int* launches)
   p.bwd_units_det = reinterpret_cast<int32_t*>(ws + l.bwd_units_det);
   p.Hkv = plan->prob.num_kv_heads;
   p.key_end = reinterpret_cast<int32_t*>(ws + l.key_end);
+  {
+    // a third of the SMs (the backward runs one CTA per SM), at most 48 tiles = 6144 tokens
+    static DeviceSetup setup[kMaxDevices];
+    DeviceSetup* dev = device_setup(setup);
+    p.det_asc_max = dev ? std::min(48, dev->num_sms / 3) : 0;
+  }
   p.num_rows = plan->prob.num_rows;
   p.G = plan->prob.num_groups;
   p.N = plan->prob.num_responses;

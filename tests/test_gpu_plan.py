@@ -77,7 +77,8 @@ def test_plan_matches_dense_mask(w, desc_on_device):
     assert len(btiles) == sum((hi - lo + 127) // 128 for lo, hi in groups.values())
     bcov = np.zeros(T, dtype=int)
     prompt_len = {s0: l0 for (s0, l0, _r, _g, k) in segs if k == 0}   # by group start
-    for (start, ln, vis_end, full_end, gstart, gend, work, npc) in btiles.tolist():
+    bt_start = {int(b[0]): i for i, b in enumerate(btiles.tolist())}
+    for (start, ln, vis_end, dep_lo, gstart, gend, work, npc) in btiles.tolist():
         assert npc == (prompt_len[gstart] + 127) // 128
         assert 1 <= ln <= 128 and (start - gstart) % 128 == 0 and start + ln <= gend
         assert ln == 128 or start + ln == gend
@@ -90,9 +91,13 @@ def test_plan_matches_dense_mask(w, desc_on_device):
         for c in range(ln):
             q = np.nonzero(cols[:, c])[0]
             assert q[0] == start + c and q[-1] + 1 == key_end[start + c] and len(q) == key_end[start + c] - start - c
-        assert vis_end == key_end[start:start + ln].max() and full_end == key_end[start:start + ln].min()
-        # queries in [start + ln, full_end) see every key of the tile
-        assert cols[start + ln:full_end].all()
+        assert vis_end == key_end[start:start + ln].max()
+        # read as a query tile: the key tiles of the group whose keys some row of this tile sees
+        # are the prompt tiles [0, npc) (up to the tile itself) and the tiles [dep_lo, own index]
+        k_rel = (start - gstart) // 128
+        seen_tiles = {kk for kk in range(k_rel + 1)
+                      if mask[start:start + ln, gstart + 128 * kk:min(gstart + 128 * kk + 128, gend)].any()}
+        assert seen_tiles == set(range(min(npc, k_rel + 1))) | set(range(dep_lo, k_rel + 1))
         assert work == 1 + (vis_end - start - ln + 127) // 128
     assert (bcov == 1).all()
     # column form of the mask: key j is visible to queries [j, key_end[j])
