@@ -4,7 +4,7 @@
 //   warp 0      TMA producer: draws and decodes the work units (the only reader of the plan's
 //               tile list; the other roles get a decoded record through shared memory), loads
 //               the Q tiles of the unit's two query heads, then the K / V tiles of every
-//               visible key tile through two-stage rings
+//               visible key tile in two-deep stages {V(j), K(j + 1)} (one barrier pair each)
 //   warp 1      MMA issuer (one thread): S = Q K^T and O += P V with tcgen05.mma, fp32 in TMEM
 //   warps 2-9   softmax warps of slot 0: two threads per query row (= TMEM lane), 64 key
 //               columns each
@@ -45,9 +45,9 @@ constexpr float kRescaleThreshold = 8.f;  // log2 units
 enum FwdBar : int {
   kQFull = 0,   // [2] per slot
   kQEmpty = 2,  // [2]
-  kKFull = 4,   // [2] per stage
-  kKEmpty = 6,
-  kVFull = 8,
+  kKFull = 4,   // [2] per K / V stage: full
+  kKEmpty = 6,  // [2]                 empty
+  kVFull = 8,   // (unused)
   kVEmpty = 10,
   kSFull = 12,  // [2] per slot
   kPFull = 14,
@@ -205,7 +205,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      uint32_t kc = 0, vc = 0, qc[2] = {0, 0};
+      uint32_t kc = 0, qc[2] = {0, 0};
       Unit un;
       for (uint32_t un_i = 0; fetch_unit(un_i, un); ++un_i) {
         for (int s = 0; s < un.nslots; ++s) {
@@ -216,33 +216,32 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                         un.tile.start, bar(kQFull + s));
           ++qc[s];
         }
-        // K runs one tile ahead of V: K(j+1) only needs QK(j-1) to be done, V(j) needs PV(j-2),
-        // so a V load waiting for its stage must not hold back the next K load.
-        auto load_k = [&](int j) {
-          const KvTile kt = kv_tile_of(un.tile, j, un.n0, un.n1);
+        // K and V travel in stages {V(j), K(j + 1)} -- what one period of the MMA thread
+        // consumes -- with ONE full / empty barrier pair per stage (the first stage of a unit
+        // holds only K(0), the last only V(last)): every barrier operation costs the MMA
+        // thread 100 - 150 cycles of tensor-pipe time, so it gets one wait and one commit per
+        // period instead of two of each.  Stage n uses the K and V buffers n & 1.
+        auto load_stage = [&](int jv, int jk) {   // key tile of V and of K in this stage, or -1
           const uint32_t st = kc & 1;
           wait_bar(bar(kKEmpty + st), ((kc >> 1) & 1) ^ 1, abort_flag, prm.header, 22);
-          mbar_expect_tx(bar(kKFull + st), L::kTileBytes);
-          for (int b = 0; b < D / 64; ++b)
-            tma_load_3d(sK + st * L::kTileBytes + b * kBoxBytes, &tm_k, b * 64, un.kvh, kt.start,
-                        bar(kKFull + st));
+          mbar_expect_tx(bar(kKFull + st), (jv >= 0 && jk >= 0 ? 2 : 1) * L::kTileBytes);
+          if (jk >= 0) {
+            const KvTile kt = kv_tile_of(un.tile, jk, un.n0, un.n1);
+            for (int b = 0; b < D / 64; ++b)
+              tma_load_3d(sK + st * L::kTileBytes + b * kBoxBytes, &tm_k, b * 64, un.kvh, kt.start,
+                          bar(kKFull + st));
+          }
+          if (jv >= 0) {
+            const KvTile kt = kv_tile_of(un.tile, jv, un.n0, un.n1);
+            for (int b = 0; b < D / 64; ++b)
+              tma_load_3d(sV + st * L::kTileBytes + b * kBoxBytes, &tm_v, b * 64, un.kvh, kt.start,
+                          bar(kKFull + st));
+          }
           ++kc;
         };
-        auto load_v = [&](int j) {
-          const KvTile kt = kv_tile_of(un.tile, j, un.n0, un.n1);
-          const uint32_t st = vc & 1;
-          wait_bar(bar(kVEmpty + st), ((vc >> 1) & 1) ^ 1, abort_flag, prm.header, 23);
-          mbar_expect_tx(bar(kVFull + st), L::kTileBytes);
-          for (int b = 0; b < D / 64; ++b)
-            tma_load_3d(sV + st * L::kTileBytes + b * kBoxBytes, &tm_v, b * 64, un.kvh, kt.start,
-                        bar(kVFull + st));
-          ++vc;
-        };
-        load_k(0);
-        for (int j = 0; j < un.ntiles && !*abort_flag; ++j) {
-          if (j + 1 < un.ntiles) load_k(j + 1);
-          load_v(j);
-        }
+        load_stage(-1, 0);
+        for (int j = 0; j < un.ntiles && !*abort_flag; ++j)
+          load_stage(j, j + 1 < un.ntiles ? j + 1 : -1);
       }
     }
   } else if (warp == 1) {
@@ -253,7 +252,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     // descriptors precomputed, barrier addresses and parities kept in registers, one branch
     // for the common case of full 128-key tiles).
     if (lane == 0) {
-      uint32_t kc = 0, vc = 0, tc0 = 0, tc1 = 0, uc0 = 0, uc1 = 0;
+      uint32_t kc = 0, tc0 = 0, tc1 = 0, uc0 = 0, uc1 = 0;
       constexpr uint32_t idesc_o = make_idesc(128, D, 0, 1);
       constexpr uint32_t idesc_full = make_idesc(128, 128, 0, 0);
       constexpr uint64_t kStageStep = uint64_t(L::kTileBytes >> 4);
@@ -275,7 +274,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         }
         mma_commit(bar(kSFull + s));
       };
-      auto issue_pv = [&](int s, uint32_t vstage, int k_len, bool first) {
+      auto issue_pv = [&](int s, uint32_t vstage, int k_len, bool first, bool last) {
         const uint64_t b = dv0 + vstage * kStageStep;
         const uint32_t tS = tmem + s * 128, tO = tmem + 256 + s * 128;
         if (k_len == kTile && !first) {
@@ -290,7 +289,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
               mma_ts(tO, tS + (kk < 4 ? kk * 8 : 64 + (kk - 4) * 8), b + mnmajor_off(kk), idesc_o,
                      !first || (kk > 0));
         }
-        mma_commit(bar(kODone + s));
+        // the accumulator is only waited for after the unit's last PV (the lazy rescale, rare,
+        // runs after S of the next tile is complete, whose commit covers this PV as well)
+        if (last) mma_commit(bar(kODone + s));
       };
       for (uint32_t un_i = 0;; ++un_i) {
         PP_TAKE_UNIT(un_i, false)
@@ -312,14 +313,13 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         for (int j = 0; j < u_ntiles; ++j) {
           const bool has_next = j + 1 < u_ntiles;
           const int nx_len = has_next ? u_klen(j + 1) : 0;
-          const uint32_t vst = vc & 1, kst = kc & 1;
-          wait_bar(bar(kVFull + vst), (vc >> 1) & 1, abort_flag, prm.header, 33);
-          if (has_next) wait_bar(bar(kKFull + kst), (kc >> 1) & 1, abort_flag, prm.header, 34);
+          const uint32_t vst = kc & 1, kst = kc & 1;   // stage {V(j), K(j + 1)}
+          wait_bar(bar(kKFull + kst), (kc >> 1) & 1, abort_flag, prm.header, 33);
           // slot 0
           wait_bar(bar(kPFull + 0), tc0 & 1, abort_flag, prm.header, 35);
           if (j == 0) wait_bar(bar(kOFree + 0), (uc0 & 1) ^ 1, abort_flag, prm.header, 37);
           tc_fence_after();
-          issue_pv(0, vst, cur_len, j == 0);
+          issue_pv(0, vst, cur_len, j == 0, !has_next);
           ++tc0;
           if (has_next) {
             issue_qk(0, kst, nx_len);
@@ -329,19 +329,15 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             wait_bar(bar(kPFull + 1), tc1 & 1, abort_flag, prm.header, 36);
             if (j == 0) wait_bar(bar(kOFree + 1), (uc1 & 1) ^ 1, abort_flag, prm.header, 38);
             tc_fence_after();
-            issue_pv(1, vst, cur_len, j == 0);
+            issue_pv(1, vst, cur_len, j == 0, !has_next);
             ++tc1;
             if (has_next) {
               issue_qk(1, kst, nx_len);
               if (j + 2 == u_ntiles) mma_commit(bar(kQEmpty + 1));
             }
           }
-          mma_commit(bar(kVEmpty + vst));
-          ++vc;
-          if (has_next) {
-            mma_commit(bar(kKEmpty + kst));
-            ++kc;
-          }
+          mma_commit(bar(kKEmpty + kst));
+          ++kc;
           cur_len = nx_len;
         }
         ++uc0;
@@ -390,7 +386,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const uint32_t tS = lane_base + s * 128 + half * 64;   // my S columns; P goes to their start
     const uint32_t tO = lane_base + 256 + s * 128 + half * (D / 2);
     float* xch = reinterpret_cast<float*>(gbase + L::kXch) + s * 512;  // [2 buffers][128 rows][2]
-    uint32_t tcS = 0;
+    uint32_t tcS = 0, ucS = 0;
     for (uint32_t un_i = 0;; ++un_i) {
       PP_TAKE_UNIT(un_i, true)
       if (u_nslots == 0) break;
@@ -486,8 +482,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           const bool need = row < u_len && (m_new - m_used) > kRescaleThreshold;
           if (!__any_sync(0xffffffffu, need)) break;  // same rows, same values in the partner warp
           const float alpha = ex2(m_used - m_new);
-          wait_bar(bar(kODone + s), (tcS - 1) & 1, abort_flag, prm.header, 42 + s);
-          tc_fence_after();
+          // PV of the previous tile is complete: the commit that announced this tile's S was
+          // issued after it and covers every earlier MMA of the issuing thread
 #pragma unroll 1
           for (int c = 0; c < D / 16; ++c) {  // eight columns at a time
             uint32_t w[8];
@@ -513,7 +509,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       xb[half] = l_part;
       named_barrier_sync(bar_id, 64);
       const float l_run = l_part + xb[half ^ 1];
-      wait_bar(bar(kODone + s), (tcS - 1) & 1, abort_flag, prm.header, 44 + s);
+      wait_bar(bar(kODone + s), ucS & 1, abort_flag, prm.header, 44 + s);
+      ++ucS;
       tc_fence_after();
       const float inv_l = 1.f / l_run;
       uint32_t ob[D / 4];
