@@ -438,7 +438,68 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         // more than the rescale threshold (rare) is the accumulator rescaled and the tile redone
         // from the S values, which stay in tensor memory until P is stored.
         uint32_t pk[32];
-        float rs;
+        float rs = 0.f;
+        bool done = false;
+        if (j > 0) {
+          // Common path (every tile but a unit's first, whose exact row maximum is formed first
+          // below -- with a guessed reference the largest P of a row would not be exactly 1,
+          // and rows that see one or two keys would lose the exact cancellation in dP - Delta): the 64 scores go through in four pieces of 16, the tensor-memory load
+          // of the next piece in flight under the exponentials of this one, and no maximum is
+          // formed from the scores: the largest exponential tells as well whether the row has
+          // outgrown its reference maximum by more than the rescale threshold
+          // (p > 2^threshold), and its max3 rides in the MUFU-bound loop for free.  (Measured:
+          // loads and the two maxima were 430 of a tile's 1850 softmax cycles, none of it
+          // overlapped with the exponentials.)
+          const float neg_m = -m_used;
+          const uint64_t sc2 = pack2(prm.scale_log2, prm.scale_log2), nm2 = pack2(neg_m, neg_m);
+          uint64_t sum2 = pack2(0.f, 0.f);
+          float pm0 = 0.f, pm1 = 0.f;
+          uint32_t wa[16], wb[16];
+          auto exp16 = [&](const uint32_t (&w)[16], int piece, auto masked_c) {
+            constexpr bool kMasked = decltype(masked_c)::value;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              float x0, x1;
+              unpack2(fma2(pack2(__uint_as_float(w[2 * i]), __uint_as_float(w[2 * i + 1])), sc2, nm2), x0, x1);
+              float p0 = ex2(x0), p1 = ex2(x1);
+              if (kMasked) {   // columns at and past col_lim are not visible
+                p0 = (16 * piece + 2 * i < col_lim) ? p0 : 0.f;
+                p1 = (16 * piece + 2 * i + 1 < col_lim) ? p1 : 0.f;
+              }
+              sum2 = add2(sum2, pack2(p0, p1));
+              if (i & 1) pm1 = max3(pm1, p0, p1); else pm0 = max3(pm0, p0, p1);
+              pk[8 * piece + i] = pack_bf16(p0, p1);
+            }
+          };
+          auto pieces = [&](auto masked_c) {
+            tmem_ld16(tS, wa);
+            tmem_wait_ld();
+            tmem_ld16(tS + 16, wb);
+            exp16(wa, 0, masked_c);
+            tmem_wait_ld();
+            tmem_ld16(tS + 32, wa);
+            exp16(wb, 1, masked_c);
+            tmem_wait_ld();
+            tmem_ld16(tS + 48, wb);
+            exp16(wa, 2, masked_c);
+            tmem_wait_ld();
+            exp16(wb, 3, masked_c);
+          };
+          if (full) pieces(std::false_type{}); else pieces(std::true_type{});
+          float s0, s1;
+          unpack2(sum2, s0, s1);
+          rs = s0 + s1;
+          const float pmax = fmaxf(pm0, pm1);
+          xb[half] = pmax;
+          named_barrier_sync(bar_id, 64);
+          const float hi = fmaxf(pmax, xb[half ^ 1]);
+          // (rows past the tile's end must not steer the warp-wide decision)
+          const bool need = row < u_len && !(hi <= exp2f(kRescaleThreshold));
+          if (!__any_sync(0xffffffffu, need)) done = true;   // same rows and values in the partner warp
+          else xb = xch + ((tcS & 1) ^ 1) * 256 + row * 2;   // rare: the exact path below, which
+                                                            // exchanges again, in the other buffer
+        }
+        if (!done)
         for (;;) {
           const float neg_m = -m_used;
           const uint64_t sc2 = pack2(prm.scale_log2, prm.scale_log2), nm2 = pack2(neg_m, neg_m);
