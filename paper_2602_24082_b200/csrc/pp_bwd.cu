@@ -411,11 +411,23 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           wait_bar(bar(kPReady), par, abort_flag, prm.header, 64);
           if (it == 0) wait_bar(bar(kDkvFree), (ucnt & 1) ^ 1, abort_flag, prm.header, 65);
           tc_fence_after();
+          // (the k-step count and the accumulate flag are decided once per group: a branch or
+          // a run-time predicate in front of every MMA costs the issuing thread more than the
+          // MMA takes)
+          auto issue_dv = [&](auto full_c, auto acc_c) {
 #pragma unroll
-          for (int k = 0; k < 8; ++k)
-            if (k < qsteps)
-              mma_ts(tmem + tdV, tmem + tS + (k < 4 ? k * 8 : 64 + (k - 4) * 8),
-                     ddo_mn + mnmajor_off(k), idesc_kv, (it > 0) || (k > 0));
+            for (int k = 0; k < 8; ++k)
+              if (decltype(full_c)::value || k < qsteps)
+                mma_ts(tmem + tdV, tmem + tS + (k < 4 ? k * 8 : 64 + (k - 4) * 8),
+                       ddo_mn + mnmajor_off(k), idesc_kv, (decltype(acc_c)::value || k > 0) ? 1u : 0u);
+          };
+          if (qsteps == 8) {
+            if (it > 0) issue_dv(std::true_type{}, std::true_type{});
+            else issue_dv(std::true_type{}, std::false_type{});
+          } else {
+            if (it > 0) issue_dv(std::false_type{}, std::true_type{});
+            else issue_dv(std::false_type{}, std::false_type{});
+          }
           mma_commit(bar(kDoEmpty));
           // S^T(it+1) = K Q^T
           QTile nx = qt;
@@ -430,16 +442,31 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           // dQ(it) = dS K, then dK += dS^T Q
           wait_bar(bar(kDsReady), par, abort_flag, prm.header, 67);
           tc_fence_after();
+          if (ksteps == 8) {
 #pragma unroll
-          for (int k = 0; k < 8; ++k)
-            if (k < ksteps)
+            for (int k = 0; k < 8; ++k)
               mma_ss(tmem + tdP, dS_mn + mnmajor_off(k), dK_mn + mnmajor_off(k), idesc_dq, k > 0);
-          mma_commit(bar(kDqFull));
+          } else {
 #pragma unroll
-          for (int k = 0; k < 8; ++k)
-            if (k < qsteps)
-              mma_ss(tmem + tdK, dS_k + kmajor_off(k), dq_mn + mnmajor_off(k), idesc_kv,
-                     (it > 0) || (k > 0));
+            for (int k = 0; k < 8; ++k)
+              if (k < ksteps)
+                mma_ss(tmem + tdP, dS_mn + mnmajor_off(k), dK_mn + mnmajor_off(k), idesc_dq, k > 0);
+          }
+          mma_commit(bar(kDqFull));
+          auto issue_dk = [&](auto full_c, auto acc_c) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              if (decltype(full_c)::value || k < qsteps)
+                mma_ss(tmem + tdK, dS_k + kmajor_off(k), dq_mn + mnmajor_off(k), idesc_kv,
+                       (decltype(acc_c)::value || k > 0) ? 1u : 0u);
+          };
+          if (qsteps == 8) {
+            if (it > 0) issue_dk(std::true_type{}, std::true_type{});
+            else issue_dk(std::true_type{}, std::false_type{});
+          } else {
+            if (it > 0) issue_dk(std::false_type{}, std::true_type{});
+            else issue_dk(std::false_type{}, std::false_type{});
+          }
           mma_commit(bar(kQEmptyB + st));
           qt = nx;
         }
