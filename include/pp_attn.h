@@ -149,7 +149,7 @@ int pp_plan_read(const pp_plan* plan, pp_stream_t stream, int32_t* num_tiles, in
  * pp_attn_bwd as its scratch (256-byte aligned, at least the backward size reported by
  * pp_plan_workspace_bytes; PP_ERR_WORKSPACE_TOO_SMALL / PP_ERR_ALIGNMENT otherwise): the
  * forward then also clears the fp32 dQ accumulator inside it (when that accumulator,
- * 4 * T * Hq * D bytes, is at most 320 MiB -- beyond that the library leaves the clearing to
+ * 4 * T * Hq * D bytes, is at most 640 MiB -- beyond that the library leaves the clearing to
  * the backward, which measured faster), and the next pp_attn_bwd on this plan with the same
  * buffer (later on the same stream) skips its own clearing pass.  The buffer must not be used
  * for anything else in between.

@@ -282,10 +282,11 @@ int pp_attn_fwd(const pp_plan* plan, const void* q, const void* k, const void* v
   // Optional: the buffer the caller will hand to pp_attn_bwd as scratch.  The forward then
   // also clears the fp32 dQ accumulator inside it (the kernel is compute-bound and has memory
   // bandwidth to spare), and the backward's preprocess pass skips its own clearing.
-  // Measured: it pays while the accumulator is a few hundred MB (0.15-0.3 GB: step -4..5 %);
-  // at 1 GB the extra stores slow the forward's loads and the zeros have left L2 long before
-  // the backward adds to them (step +2 %), so larger accumulators are left to the backward.
-  constexpr size_t kFwdClearMaxBytes = size_t(320) << 20;
+  // Measured: it pays while the accumulator is a few hundred MB (0.15-0.3 GB: step -4..5 %,
+  // 0.54 GB: -1.5..4 %); at 1 GB the extra stores slow the forward's loads and the zeros have
+  // left L2 long before the backward adds to them (step +2 %), so larger accumulators are left
+  // to the backward.
+  constexpr size_t kFwdClearMaxBytes = size_t(640) << 20;
   float* dq_clear = nullptr;
   plan->cleared_scratch = nullptr;
   if (d_scratch) {
