@@ -407,6 +407,16 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
               mma_ss(tmem + tdP, dV_k + kmajor_off(k), ddo_k + kmajor_off(k), idesc, k > 0);
             mma_commit(bar(kDpFull));
           }
+          // (the next tile's coordinates and descriptors are worked out here, while the pipe is
+          // still busy with dP, not between dV and S)
+          QTile nx = qt;
+          const bool has_next = it + 1 < un.n_it;
+          if (has_next) {
+            q_advance(qi, prm.Hq / prm.Hkv);
+            nx = q_tile_at(prm, un, qi);
+          }
+          const uint32_t idesc_s_next = make_idesc(128, ((nx.len + 15) >> 4) << 4, 0, 0);
+          const uint64_t dq_k_next = kmajor_base(sQ) + ((g + 1) & 1) * kStageStep;
           // dV += P^T dO
           wait_bar(bar(kPReady), par, abort_flag, prm.header, 64);
           if (it == 0) wait_bar(bar(kDkvFree), (ucnt & 1) ^ 1, abort_flag, prm.header, 65);
@@ -430,14 +440,14 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           }
           mma_commit(bar(kDoEmpty));
           // S^T(it+1) = K Q^T
-          QTile nx = qt;
-          if (it + 1 < un.n_it) {
-            q_advance(qi, prm.Hq / prm.Hkv);
-            nx = q_tile_at(prm, un, qi);
+          if (has_next) {
             const uint32_t g1 = g + 1;
             wait_bar(bar(kQFullB + (g1 & 1)), (g1 >> 1) & 1, abort_flag, prm.header, 66);
             tc_fence_after();
-            issue_s(g1 & 1, nx.len);
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k)
+              mma_ss(tmem + tS, dK_k + kmajor_off(k), dq_k_next + kmajor_off(k), idesc_s_next, k > 0);
+            mma_commit(bar(kSFullB));
           }
           // dQ(it) = dS K, then dK += dS^T Q
           wait_bar(bar(kDsReady), par, abort_flag, prm.header, 67);
