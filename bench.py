@@ -460,6 +460,37 @@ class Runner:
             "tflops": b_flops / (statistics.median(dms) * 1e-3) / 1e12,
             "slowdown": statistics.median(dms) / statistics.median(nms)}
 
+        # ---- next row: head_dim 96 (the same packing structure and head counts; the kernels run
+        # it in tiles of 128 columns whose upper quarter the TMA loads fill with zeros)
+        from paper_2602_24082_b200 import workloads as W96
+        w96 = W96.Workload(w.name + "-d96", w.rows, Hq, Hkv, 96, seed=96)
+        q9, k9, v9, do9 = (x.to(dev) for x in w96.tensors())
+        plan9 = B.plan_for(w96, desc_on_device=True)
+        f9, b9 = w96.useful_flops()
+        o9 = lse9 = None
+        for _ in range(3):
+            o9, lse9 = B.pp_attn_fwd(plan9, q9, k9, v9, w96.softmax_scale)
+            B.pp_attn_bwd(plan9, q9, k9, v9, o9, lse9, do9, w96.softmax_scale)
+        fms, bms = [], []
+        for _ in range(5):
+            self.flush.zero_()
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            ev[0].record()
+            o9, lse9 = B.pp_attn_fwd(plan9, q9, k9, v9, w96.softmax_scale)
+            ev[1].record()
+            B.pp_attn_bwd(plan9, q9, k9, v9, o9, lse9, do9, w96.softmax_scale)
+            ev[2].record()
+            torch.cuda.synchronize()
+            fms.append(ev[0].elapsed_time(ev[1]))
+            bms.append(ev[1].elapsed_time(ev[2]))
+        fm, bm = statistics.median(fms), statistics.median(bms)
+        out["head_dim_96"] = {"fwd_ms": fm, "bwd_ms": bm,
+                              "fwd_tflops": f9 / (fm * 1e-3) / 1e12,
+                              "bwd_tflops": b9 / (bm * 1e-3) / 1e12,
+                              "value": (f9 + b9) / ((fm + bm) * 1e-3) / 1e12, "unit": "TFLOP/s",
+                              "note": "forward + backward (preprocess, main, finalize), plan excluded"}
+        del q9, k9, v9, do9, o9, lse9, plan9
+
         # ---- next row: the row builder (batch sorting + packing into rows) on a synthetic
         # batch of 4096 preference groups of up to 16K tokens, rows of 16384 tokens, and the
         # assignment of those rows to 8 data-parallel ranks

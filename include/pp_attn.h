@@ -39,7 +39,7 @@ enum pp_status {
   PP_OK = 0,
   PP_ERR_INVALID_ARG = -1,         /* null pointer, non-positive length, non-monotone offsets,
                                       total_tokens mismatch, Hq % Hkv != 0 */
-  PP_ERR_UNSUPPORTED = -2,         /* head_dim not in {64, 128}; device is not compute capability 10.x */
+  PP_ERR_UNSUPPORTED = -2,         /* head_dim not in {64, 96, 128}; device is not compute capability 10.x */
   PP_ERR_WORKSPACE_TOO_SMALL = -3, /* plan workspace or scratch smaller than the size query says */
   PP_ERR_ALIGNMENT = -4,           /* a tensor base pointer is not 16-byte aligned */
   PP_ERR_CUDA = -5,                /* a CUDA runtime / driver call failed */
@@ -67,7 +67,7 @@ typedef struct {
                                     1: device arrays (validated by the plan kernel)          */
   int32_t num_q_heads;           /* Hq                                                        */
   int32_t num_kv_heads;          /* Hkv, divides Hq                                           */
-  int32_t head_dim;              /* D: 64 or 128                                              */
+  int32_t head_dim;              /* D: 64, 96 or 128                                          */
   int32_t total_tokens;          /* T = sum of every prompt and response length (checked)     */
 } pp_problem;
 

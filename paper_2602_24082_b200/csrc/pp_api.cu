@@ -66,7 +66,7 @@ int check_problem_shape(const pp_problem* p) {
   if (p->num_groups < p->num_rows || p->num_responses < p->num_groups) return PP_ERR_INVALID_ARG;
   if (p->num_q_heads < 1 || p->num_kv_heads < 1 || p->num_q_heads % p->num_kv_heads != 0)
     return PP_ERR_INVALID_ARG;
-  if (p->head_dim != 64 && p->head_dim != 128) return PP_ERR_UNSUPPORTED;
+  if (p->head_dim != 64 && p->head_dim != 96 && p->head_dim != 128) return PP_ERR_UNSUPPORTED;
   // unit records pack (kv head << 24) | tile
   if (p->num_kv_heads > 127 || p->total_tokens / 128 + p->num_groups + p->num_responses >= (1 << 24))
     return PP_ERR_UNSUPPORTED;

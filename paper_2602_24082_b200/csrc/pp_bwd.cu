@@ -48,12 +48,15 @@ struct BwdParams {
 // second measured about 5 us faster where a token's heads span 8 KB (Hq = 32, D = 128,
 // T = 9241), the first about 60 us faster at 16 KB (Hq = 64, T = 16384); the launcher picks by
 // that size.
+// lanes that share a row: D / 8 (16 bytes of bf16 per lane), rounded up to a power of two
+__host__ __device__ constexpr int pre_lanes(int d) { return d == 96 ? 16 : d / 8; }
+
 template <int D, bool kClear, bool kTokenMajor>
 __global__ void __launch_bounds__(256)
 bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
                       const float* __restrict__ lse, float* __restrict__ delta,
                       float* __restrict__ lse2, float* __restrict__ dq_acc, int T, int Hq) {
-  constexpr int kLanes = D / 8;           // lanes per row
+  constexpr int kLanes = pre_lanes(D);    // lanes per row (D / 8 of them hold data)
   constexpr int kRows = 32 / kLanes;      // rows per warp and step
   constexpr int kUnroll = 4;
   const int lane = threadIdx.x & 31, sub = lane % kLanes, rin = lane / kLanes;
@@ -68,7 +71,7 @@ bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* 
       // written to consecutive addresses (each O / dO row is one contiguous piece anyway)
       const long long idx = base + u * kRows + rin;
       a[u] = b[u] = make_uint4(0u, 0u, 0u, 0u);
-      if (idx < rows) {
+      if (idx < rows && sub < D / 8) {
         long long row = idx;
         if (!kTokenMajor) {
           const int h = int(idx / T), t = int(idx - (long long)h * T);
@@ -100,7 +103,7 @@ bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* 
           const int h = int(idx / T), t = int(idx - (long long)h * T);
           row = (long long)t * Hq + h;
         }
-        if (kClear) {
+        if (kClear && sub < D / 8) {
           float4* z = reinterpret_cast<float4*>(dq_acc + row * D + sub * 8);
           z[0] = make_float4(0.f, 0.f, 0.f, 0.f);
           z[1] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -232,7 +235,10 @@ __device__ __forceinline__ QTile q_tile_at(const BwdParams& prm, const BwdUnit& 
   return q;
 }
 
-template <int D, bool kDet>
+// D: head dimension of the shared-memory tiles; DV <= D: head dimension of the tensors in
+// global memory (96 in tiles of 128: the TMA loads zero-fill the columns past DV, so only the
+// loops over the head dimension, the N of dV / dK / dQ and global addressing know about DV).
+template <int D, bool kDet, int DV = D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
            const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
@@ -369,8 +375,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       uint32_t gc = 0, ucnt = 0;
-      constexpr uint32_t idesc_kv = make_idesc(128, D, 0, 1);  // dV, dK : K-major A, MN-major B
-      constexpr uint32_t idesc_dq = make_idesc(128, D, 1, 1);  // dQ     : MN-major A and B
+      constexpr uint32_t idesc_kv = make_idesc(128, DV, 0, 1);  // dV, dK : K-major A, MN-major B
+      constexpr uint32_t idesc_dq = make_idesc(128, DV, 1, 1);  // dQ     : MN-major A and B
       BwdUnit un;
       const uint64_t dK_k = kmajor_base(sK), dV_k = kmajor_base(sV), dK_mn = mnmajor_base(sK);
       const uint64_t dS_k = kmajor_base(sdS), dS_mn = mnmajor_base(sdS);
@@ -379,7 +385,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         const uint32_t idesc = make_idesc(128, ((q_len + 15) >> 4) << 4, 0, 0);
         const uint64_t dq_k = kmajor_base(sQ) + st * kStageStep;
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k)
+        for (int k = 0; k < DV / 16; ++k)
           mma_ss(tmem + tS, dK_k + kmajor_off(k), dq_k + kmajor_off(k), idesc, k > 0);
         mma_commit(bar(kSFullB));
       };
@@ -403,7 +409,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           {
             const uint32_t idesc = make_idesc(128, qsteps << 4, 0, 0);
 #pragma unroll
-            for (int k = 0; k < D / 16; ++k)
+            for (int k = 0; k < DV / 16; ++k)
               mma_ss(tmem + tdP, dV_k + kmajor_off(k), ddo_k + kmajor_off(k), idesc, k > 0);
             mma_commit(bar(kDpFull));
           }
@@ -445,7 +451,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             wait_bar(bar(kQFullB + (g1 & 1)), (g1 >> 1) & 1, abort_flag, prm.header, 66);
             tc_fence_after();
 #pragma unroll
-            for (int k = 0; k < D / 16; ++k)
+            for (int k = 0; k < DV / 16; ++k)
               mma_ss(tmem + tS, dK_k + kmajor_off(k), dq_k_next + kmajor_off(k), idesc_s_next, k > 0);
             mma_commit(bar(kSFullB));
           }
@@ -598,8 +604,13 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
         uint32_t w[32];
-        tmem_ld32(lane_base + tsrc + c * 32, w);
-        tmem_wait_ld();
+        if (DV == D || c * 32 < DV) {
+          tmem_ld32(lane_base + tsrc + c * 32, w);
+          tmem_wait_ld();
+        } else {  // columns past DV hold nothing and are not stored
+#pragma unroll
+          for (int i = 0; i < 32; ++i) w[i] = 0u;
+        }
 #pragma unroll
         for (int i = 0; i < 16; ++i)
           ob[c * 16 + i] = pack_bf16(__uint_as_float(w[2 * i]) * f, __uint_as_float(w[2 * i + 1]) * f);
@@ -641,9 +652,9 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             const int r = 32 * (warp & 3) + grp * 8 + i;
-            if (r < un.tile.len) {
+            if (r < un.tile.len && (DV == D || hb * 64 + chunk * 8 < DV)) {
               uint4* dst = reinterpret_cast<uint4*>(
-                  out + ((size_t(un.tile.start) + r) * prm.Hkv + un.kvh) * D + hb * 64 + chunk * 8);
+                  out + ((size_t(un.tile.start) + r) * prm.Hkv + un.kvh) * DV + hb * 64 + chunk * 8);
               *dst = make_uint4(ob[32 * hb + 4 * i], ob[32 * hb + 4 * i + 1], ob[32 * hb + 4 * i + 2],
                                 ob[32 * hb + 4 * i + 3]);
             }
@@ -706,9 +717,15 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         for (int half = 0; half < 2; ++half) {
           uint32_t w[D / 2];
 #pragma unroll
-          for (int c = 0; c < D / 64; ++c)
-            tmem_ld32(lane_base + tdP + half * (D / 2) + c * 32,
-                      *reinterpret_cast<uint32_t(*)[32]>(&w[c * 32]));
+          for (int c = 0; c < D / 64; ++c) {
+            if (DV == D || half * (D / 2) + c * 32 < DV) {
+              tmem_ld32(lane_base + tdP + half * (D / 2) + c * 32,
+                        *reinterpret_cast<uint32_t(*)[32]>(&w[c * 32]));
+            } else {  // no such columns in global memory: the box is not reduced either
+#pragma unroll
+              for (int i = 0; i < 32; ++i) w[c * 32 + i] = 0u;
+            }
+          }
           tmem_wait_ld();
           if (half == 1) {
             tc_fence_before();
@@ -763,7 +780,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                   *abort_flag = 1;
                 }
               }
-              tma_reduce_add_3d(&tm_dq, buf, half * (D / 2) + c * 32, qt.h, qt.start);
+              if (DV == D || half * (D / 2) + c * 32 < DV)
+                tma_reduce_add_3d(&tm_dq, buf, half * (D / 2) + c * 32, qt.h, qt.start);
               bulk_commit_group();
             }
           }
@@ -824,7 +842,7 @@ namespace pp {
 namespace {
 #endif
 
-template <int D>
+template <int D, int DV = D>
 cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, const void* d_o,
                          void* dq, const CUtensorMap& tq, const CUtensorMap& tk,
                          const CUtensorMap& tv, const CUtensorMap& tdo, const CUtensorMap& tdq,
@@ -834,13 +852,13 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
   DeviceSetup* dev = device_setup(setup);
   if (!dev) return cudaErrorInvalidDevice;
   if (dev->cc_major != 10) return cudaErrorNotSupported;
-  auto kern = prm.dq_sem ? bwd_kernel<D, true> : bwd_kernel<D, false>;
+  auto kern = prm.dq_sem ? bwd_kernel<D, true, DV> : bwd_kernel<D, false, DV>;
   if (!dev->configured) {
-    cudaError_t e = cudaFuncSetAttribute(bwd_kernel<D, false>,
+    cudaError_t e = cudaFuncSetAttribute(bwd_kernel<D, false, DV>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          BwdSmem<D>::kTotal);
     if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(bwd_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+      e = cudaFuncSetAttribute(bwd_kernel<D, true, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                BwdSmem<D>::kTotal);
     if (e != cudaSuccess) return e;
     dev->configured = true;
@@ -849,16 +867,16 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
   const size_t T = pb.total_tokens, Hq = pb.num_q_heads;
   const long long pairs = (long long)T * Hq;
   const int num_sms = dev->num_sms;
-  constexpr int kRowsPerBlock = 8 * (32 / (D / 8)) * 4;  // warps x rows per warp x unroll
+  constexpr int kRowsPerBlock = 8 * (32 / pre_lanes(DV)) * 4;  // warps x rows per warp x unroll
   const unsigned pre_blocks = unsigned(
       std::min<long long>((pairs + kRowsPerBlock - 1) / kRowsPerBlock, (long long)num_sms * 16));
   auto pre = [&](auto clear, auto token_major) {
-    bwd_preprocess_kernel<D, decltype(clear)::value, decltype(token_major)::value>
+    bwd_preprocess_kernel<DV, decltype(clear)::value, decltype(token_major)::value>
         <<<pre_blocks, 256, 0, stream>>>(
             static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse,
             const_cast<float*>(prm.delta), const_cast<float*>(prm.lse2), prm.dq_acc, int(T), int(Hq));
   };
-  const bool token_major = Hq * D * 2 >= 16384;
+  const bool token_major = Hq * DV * 2 >= 16384;
   if (dq_cleared) {
     if (token_major) pre(std::false_type{}, std::true_type{});
     else pre(std::false_type{}, std::false_type{});
@@ -875,7 +893,7 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
     profile_record(ev.bwd1, stream);
     ev.bwd_valid = true;
   }
-  const size_t n4 = T * Hq * D / 4;
+  const size_t n4 = T * Hq * DV / 4;
   unsigned fb = unsigned(std::min<size_t>((n4 + 255) / 256, size_t(num_sms) * 16));
   bwd_finalize_kernel<<<fb, 256, 0, stream>>>(reinterpret_cast<const float4*>(prm.dq_acc),
                                               static_cast<uint2*>(dq), n4, prm.scale);
@@ -923,11 +941,14 @@ cudaError_t launch_bwd(const pp_plan* plan, const void* q, const void* k, const 
   CUtensorMap tdq;
   if (!encode_thd_f32(&tdq, prm.dq_acc, pb.total_tokens, pb.num_q_heads, pb.head_dim))
     return cudaErrorNotSupported;
-  return pb.head_dim == 128
-             ? launch_bwd_t<128>(plan, o, lse, d_o, dq, tq, tk, tv, tdo, tdq, prm, dq_cleared, stream,
-                                 launches)
-             : launch_bwd_t<64>(plan, o, lse, d_o, dq, tq, tk, tv, tdo, tdq, prm, dq_cleared, stream,
-                                launches);
+  if (pb.head_dim == 128)
+    return launch_bwd_t<128>(plan, o, lse, d_o, dq, tq, tk, tv, tdo, tdq, prm, dq_cleared, stream,
+                             launches);
+  if (pb.head_dim == 96)
+    return launch_bwd_t<128, 96>(plan, o, lse, d_o, dq, tq, tk, tv, tdo, tdq, prm, dq_cleared,
+                                 stream, launches);
+  return launch_bwd_t<64>(plan, o, lse, d_o, dq, tq, tk, tv, tdo, tdq, prm, dq_cleared, stream,
+                          launches);
 }
 
 // ---------------------------------------------------------------- built-in scratch

@@ -117,7 +117,11 @@ __device__ __forceinline__ bool get_unit(const FwdParams& prm, int u, int ntiles
   return true;
 }
 
-template <int D>
+// D: head dimension of the shared-memory tiles (64 or 128); DV <= D: head dimension of the
+// tensors in global memory.  For DV < D (96 in tiles of 128) the TMA loads fill the columns
+// past DV with zeros, so only the loops over the head dimension, the N of the second GEMM and
+// everything that addresses global memory know about DV.
+template <int D, int DV = D>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
            const __grid_constant__ CUtensorMap tm_v, FwdParams prm) {
@@ -253,7 +257,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     // for the common case of full 128-key tiles).
     if (lane == 0) {
       uint32_t kc = 0, tc0 = 0, tc1 = 0, uc0 = 0, uc1 = 0;
-      constexpr uint32_t idesc_o = make_idesc(128, D, 0, 1);
+      constexpr uint32_t idesc_o = make_idesc(128, DV, 0, 1);
       constexpr uint32_t idesc_full = make_idesc(128, 128, 0, 0);
       constexpr uint64_t kStageStep = uint64_t(L::kTileBytes >> 4);
       const uint64_t dq0 = kmajor_base(sQ), dk0 = kmajor_base(sK), dv0 = mnmajor_base(sV);
@@ -264,12 +268,12 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         const uint32_t tS = tmem + s * 128;
         if (k_len == kTile) {
 #pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk)
+          for (int kk = 0; kk < DV / 16; ++kk)
             mma_ss(tS, a + kmajor_off(kk), b + kmajor_off(kk), idesc_full, kk > 0);
         } else {
           const uint32_t idesc_s = make_idesc(128, 0, 0, 0) | (uint32_t(((k_len + 15) >> 4) << 1) << 17);
 #pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk)
+          for (int kk = 0; kk < DV / 16; ++kk)
             mma_ss(tS, a + kmajor_off(kk), b + kmajor_off(kk), idesc_s, kk > 0);
         }
         mma_commit(bar(kSFull + s));
@@ -356,13 +360,13 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       for (uint32_t un_i = 0;; ++un_i) {
         PP_TAKE_UNIT(un_i, true)
         if (u_nslots == 0) break;
-        constexpr int kChunks = D / 4;  // 16-byte chunks per row
+        constexpr int kChunks = DV / 4;  // 16-byte chunks per row
         const int total = u_len * kChunks;
         for (int sl = 0; sl < u_nslots; ++sl) {
-          float* base = prm.dq_clear + (size_t(u_start) * prm.Hq + (u_h0 + sl)) * D;
+          float* base = prm.dq_clear + (size_t(u_start) * prm.Hq + (u_h0 + sl)) * DV;
           for (int c = cl; c < total; c += 64) {
             const int r = c / kChunks, col = c - r * kChunks;
-            *reinterpret_cast<float4*>(base + size_t(r) * prm.Hq * D + col * 4) =
+            *reinterpret_cast<float4*>(base + size_t(r) * prm.Hq * DV + col * 4) =
                 make_float4(0.f, 0.f, 0.f, 0.f);
           }
         }
@@ -578,8 +582,14 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 #pragma unroll
       for (int c = 0; c < D / 64; ++c) {
         uint32_t w[32];
-        tmem_ld32(tO + c * 32, w);
-        tmem_wait_ld();
+        // (columns at and past DV hold nothing and are not stored: the zeros only fill ob)
+        if (DV == D || half * (D / 2) + c * 32 < DV) {
+          tmem_ld32(tO + c * 32, w);
+          tmem_wait_ld();
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) w[i] = 0u;
+        }
 #pragma unroll
         for (int i = 0; i < 16; ++i)
           ob[c * 16 + i] = pack_bf16(__uint_as_float(w[2 * i]) * inv_l, __uint_as_float(w[2 * i + 1]) * inv_l);
@@ -621,9 +631,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 #pragma unroll
         for (int i = 0; i < kCh; ++i) {
           const int r = 32 * qd + grp * kCh + i;
-          if (r < u_len) {
+          if (r < u_len && (DV == D || half * (D / 2) + chunk * 8 < DV)) {
             uint4* dst = reinterpret_cast<uint4*>(
-                prm.o + ((size_t(u_start) + r) * prm.Hq + h) * D + half * (D / 2) + chunk * 8);
+                prm.o + ((size_t(u_start) + r) * prm.Hq + h) * DV + half * (D / 2) + chunk * 8);
             *dst = make_uint4(ob[4 * i], ob[4 * i + 1], ob[4 * i + 2], ob[4 * i + 3]);
           }
         }
@@ -670,14 +680,14 @@ namespace pp {
 namespace {
 #endif
 
-template <int D>
+template <int D, int DV = D>
 cudaError_t launch_fwd_t(const pp_plan* plan, const CUtensorMap& tq, const CUtensorMap& tk,
                          const CUtensorMap& tv, const FwdParams& prm, cudaStream_t stream) {
   static DeviceSetup setup[kMaxDevices];
   DeviceSetup* dev = device_setup(setup);
   if (!dev) return cudaErrorInvalidDevice;
   if (dev->cc_major != 10) return cudaErrorNotSupported;
-  auto kern = fwd_kernel<D>;
+  auto kern = fwd_kernel<D, DV>;
   if (!dev->configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          FwdSmem<D>::kTotal);
@@ -720,8 +730,9 @@ cudaError_t launch_fwd(const pp_plan* plan, const void* q, const void* k, const 
   prm.Hq = pb.num_q_heads;
   prm.Hkv = pb.num_kv_heads;
   prm.scale_log2 = scale * 1.4426950408889634f;
-  cudaError_t e = pb.head_dim == 128 ? launch_fwd_t<128>(plan, tq, tk, tv, prm, stream)
-                                     : launch_fwd_t<64>(plan, tq, tk, tv, prm, stream);
+  cudaError_t e = pb.head_dim == 128  ? launch_fwd_t<128>(plan, tq, tk, tv, prm, stream)
+                  : pb.head_dim == 96 ? launch_fwd_t<128, 96>(plan, tq, tk, tv, prm, stream)
+                                      : launch_fwd_t<64>(plan, tq, tk, tv, prm, stream);
   if (e == cudaSuccess && launches) *launches += 1;
   return e;
 }

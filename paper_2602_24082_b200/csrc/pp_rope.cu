@@ -62,11 +62,12 @@ rope_kernel(SegPtrs p, __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict_
   if (t >= p.T) return;
   const float pos = float(position_of(p, t));
   constexpr int kHalf = D / 2;
-  if (D == 128) {
+  if (D != 64) {   // two frequencies per lane: lanes 0 .. D / 4 - 1 cover the D / 2 pairs
     float c0, s0, c1, s1;
     sincosf(pos * exp2f(-log2_base * (2.f * float(2 * lane) / float(D))), &s0, &c0);
     sincosf(pos * exp2f(-log2_base * (2.f * float(2 * lane + 1) / float(D))), &s1, &c1);
     auto rotate = [&](__nv_bfloat16* x) {
+      if (lane >= D / 4) return;
       __nv_bfloat162* lo = reinterpret_cast<__nv_bfloat162*>(x) + lane;
       __nv_bfloat162* hi = reinterpret_cast<__nv_bfloat162*>(x + kHalf) + lane;
       const float2 a = __bfloat1622float2(*lo), b = __bfloat1622float2(*hi);
@@ -117,6 +118,10 @@ cudaError_t launch_rope(const pp_plan* plan, void* q, void* k, float base, cudaS
     rope_kernel<128><<<blocks, 256, 0, stream>>>(p, static_cast<__nv_bfloat16*>(q),
                                                  static_cast<__nv_bfloat16*>(k), pb.num_q_heads,
                                                  pb.num_kv_heads, log2_base);
+  else if (pb.head_dim == 96)
+    rope_kernel<96><<<blocks, 256, 0, stream>>>(p, static_cast<__nv_bfloat16*>(q),
+                                                static_cast<__nv_bfloat16*>(k), pb.num_q_heads,
+                                                pb.num_kv_heads, log2_base);
   else
     rope_kernel<64><<<blocks, 256, 0, stream>>>(p, static_cast<__nv_bfloat16*>(q),
                                                 static_cast<__nv_bfloat16*>(k), pb.num_q_heads,

@@ -54,7 +54,7 @@ def test_workspace_query_and_shape_errors(lib):
     plan_b, fwd_b, bwd_b = B.pp_plan_workspace_bytes(p)
     assert plan_b > 4 * w.total_tokens and fwd_b == 0
     assert bwd_b >= 4 * w.total_tokens * w.num_q_heads * (w.head_dim + 2)
-    for over, code in ((dict(head_dim=96), -2), (dict(num_kv_heads=5), -1), (dict(num_rows=0), -1),
+    for over, code in ((dict(head_dim=80), -2), (dict(head_dim=256), -2), (dict(num_kv_heads=5), -1), (dict(num_rows=0), -1),
                        (dict(total_tokens=0), -1), (dict(num_q_heads=0), -1)):
         bad, keep2 = _problem(w, **over)
         with pytest.raises(B.PPError) as e:

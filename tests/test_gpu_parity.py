@@ -83,6 +83,10 @@ RAGGED = [
     ("d128-exact-tiles", [[(256, (128, 256, 128))], [(128, (128,))]], 5, 5, 128),
     # a token's heads span 16 KB: the backward's preprocess walks memory order from there on
     ("d128-wide-heads", [[(70, (33, 129))], [(5, (64,))]], 64, 16, 128),
+    # head_dim 96 runs in tiles of 128 whose upper columns the TMA loads fill with zeros
+    ("d96-ragged", [[(257, (5, 128, 31))], [(1, (1, 300))]], 4, 2, 96),
+    ("d96-groups-gqa3", [[(97, (64, 200)), (128, (128, 128)), (3, (2, 1))], [(300, (140, 10, 129))]], 6, 2, 96),
+    ("d96-wide-heads", [[(70, (33, 129))], [(5, (64,))]], 96, 16, 96),
 ]
 
 
@@ -124,7 +128,18 @@ def test_random_structures(seed):
         assert _rel_l2(runs[0][0].float().cpu().numpy().astype(np.float64), gpu[2]) < 1e-3
 
 
-@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("seed", range(100, 112))
+def test_random_structures_head_dim_96(seed):
+    """The random structures again with head_dim 96 (tiles of 128 with zero-filled columns)."""
+    base = W.random_structure(seed, long=(seed % 4 == 0))
+    w = W.Workload(f"random-d96-{seed}", base.rows, base.num_q_heads, base.num_kv_heads, 96,
+                   seed=2000 + seed)
+    tens = w.tensors()
+    check_against_oracle(w, tens, _run_gpu(w, tens, desc_on_device=bool(seed & 1),
+                                           for_backward=bool(seed & 2)))
+
+
+@pytest.mark.parametrize("d", [64, 96, 128])
 def test_growing_scores_take_the_rescale_path(d):
     """Later keys score far higher than earlier ones (queries and keys of later token ranges are
     amplified), so a row's running maximum jumps by more than the forward's lazy-rescale
@@ -309,6 +324,7 @@ DET_CASES = [
     # groups, tiles that straddle segments: the turn order has to follow the tile order
     ("inversions", [[(200, (150, 40, 900)), (127, (1, 128)), (513, (3, 700, 2))]], 4, 2, 64),
     ("many-heads", [[(1000, (300, 500))], [(129, (640,))]], 8, 2, 128),
+    ("d96", [[(200, (150, 40, 300)), (127, (1, 128))]], 6, 2, 96),
 ]
 
 

@@ -12,6 +12,7 @@ CASES = [
     W.config0(),
     W.Workload("ragged", [[(257, (5, 128, 31))], [(1, (1, 300))]], 4, 2, 128, seed=4),
     W.Workload("groups", [[(97, (64, 200)), (128, (128, 128)), (3, (2, 1))], [(700, (1,))]], 2, 2, 64, seed=5),
+    W.Workload("d96", [[(97, (64, 200)), (3, (2, 1))], [(130, (1, 40))]], 6, 2, 96, seed=6),
 ] + [W.random_structure(s) for s in range(8)]
 
 
