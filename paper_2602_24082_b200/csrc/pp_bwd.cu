@@ -339,7 +339,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       for (int it = 0; it < un.n_it && !*abort_flag; ++it, ++qc, q_advance(qi, prm.Hq / prm.Hkv)) {
         const QTile qt = q_tile_at(prm, un, qi);
         const uint32_t st = qc & 1, par = ((qc >> 1) & 1) ^ 1;
-        // per-query statistics, fetched before the stage is known to be free;
+        // per-query statistics, fetched before the stage is known to be free and handed on
+        // NEGATED (the compute warps add them in packed two-lane instructions);
         // +inf LSE and zero Delta switch off columns past the tile's end
         const size_t row0 = size_t(qt.h) * prm.T + qt.start;
         float r_lse[4], r_del[4];
@@ -359,8 +360,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         float* sl = stats + st * 256;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          sl[lane + 32 * i] = r_lse[i];
-          sl[128 + lane + 32 * i] = r_del[i];
+          sl[lane + 32 * i] = -r_lse[i];
+          sl[128 + lane + 32 * i] = -r_del[i];
         }
         mbar_arrive(bar(kQFullB + st));
         if (lane == 0) {
@@ -527,16 +528,18 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         tmem_wait_ld();
         uint32_t pk[32];
         const float4* sl4 = reinterpret_cast<const float4*>(sl);
+        const uint64_t sc2 = pack2(prm.scale_log2, prm.scale_log2);
         if (full) {
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const float4 l = sl4[i];
-            const float p0 = ex2(fmaf(__uint_as_float(v[4 * i]), prm.scale_log2, -l.x));
-            const float p1 = ex2(fmaf(__uint_as_float(v[4 * i + 1]), prm.scale_log2, -l.y));
-            const float p2 = ex2(fmaf(__uint_as_float(v[4 * i + 2]), prm.scale_log2, -l.z));
-            const float p3 = ex2(fmaf(__uint_as_float(v[4 * i + 3]), prm.scale_log2, -l.w));
-            pk[2 * i] = pack_bf16(p0, p1);
-            pk[2 * i + 1] = pack_bf16(p2, p3);
+            const float4 l = sl4[i];   // -LSE * log2(e)
+            float x0, x1, x2, x3;
+            unpack2(fma2(pack2(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1])), sc2,
+                         pack2(l.x, l.y)), x0, x1);
+            unpack2(fma2(pack2(__uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3])), sc2,
+                         pack2(l.z, l.w)), x2, x3);
+            pk[2 * i] = pack_bf16(ex2(x0), ex2(x1));
+            pk[2 * i + 1] = pack_bf16(ex2(x2), ex2(x3));
           }
           if (!row_all) {
 #pragma unroll
@@ -548,8 +551,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             const int c0 = cb + 2 * i;
-            float p0 = ex2(fmaf(__uint_as_float(v[2 * i]), prm.scale_log2, -sl[2 * i]));
-            float p1 = ex2(fmaf(__uint_as_float(v[2 * i + 1]), prm.scale_log2, -sl[2 * i + 1]));
+            float p0 = ex2(fmaf(__uint_as_float(v[2 * i]), prm.scale_log2, sl[2 * i]));
+            float p1 = ex2(fmaf(__uint_as_float(v[2 * i + 1]), prm.scale_log2, sl[2 * i + 1]));
             p0 = (c0 >= lo && c0 < hi) ? p0 : 0.f;
             p1 = (c0 + 1 >= lo && c0 + 1 < hi) ? p1 : 0.f;
             pk[i] = pack_bf16(p0, p1);
@@ -572,9 +575,13 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           for (int i = 0; i < 16; ++i) {
             const uint32_t pp = pk[16 * half + i];
             const float p0 = __uint_as_float(pp << 16), p1 = __uint_as_float(pp & 0xffff0000u);
-            const float2 dl = reinterpret_cast<const float2*>(sl + 128 + 32 * half)[i];
-            float d0 = p0 * (__uint_as_float(d[2 * i]) - dl.x);
-            float d1 = p1 * (__uint_as_float(d[2 * i + 1]) - dl.y);
+            const float2 dl = reinterpret_cast<const float2*>(sl + 128 + 32 * half)[i];   // -Delta
+            float d0, d1;
+            unpack2(fma2(pack2(p0, p1),
+                         add2(pack2(__uint_as_float(d[2 * i]), __uint_as_float(d[2 * i + 1])),
+                              pack2(dl.x, dl.y)),
+                         pack2(0.f, 0.f)),
+                    d0, d1);
             if (!full) {  // stale tensor-memory columns may hold anything
               d0 = (pp & 0xffffu) ? d0 : 0.f;
               d1 = (pp & 0xffff0000u) ? d1 : 0.f;
