@@ -293,6 +293,17 @@ int pp_attn_step_host(const pp_problem* problem, const void* h_q, const void* h_
  */
 int pp_profile_enable(int on);
 int pp_profile_read(float* fwd_kernel_ms, float* bwd_main_kernel_ms);
+/*
+ * The same for many calls at once: the event pairs form a ring of 64 per kernel, so a benchmark
+ * can run its timed steps without a synchronisation in between and read the durations (ms,
+ * oldest first, at most `capacity` and at most 64 of the most recent launches since the last
+ * pp_profile_enable) after synchronising the stream once.  HOST arrays; either may be NULL;
+ * *num_fwd / *num_bwd receive how many entries were written.  PP_ERR_CUDA if profiling is off
+ * or an event has not completed.  Calling pp_profile_enable again while profiling is on
+ * restarts the counts.
+ */
+int pp_profile_read_all(float* fwd_kernel_ms, float* bwd_main_kernel_ms, int32_t capacity,
+                        int32_t* num_fwd, int32_t* num_bwd);
 
 /*
  * Row builder: the step before the attention path (batch sorting and batch packing, Sec. 2.2;

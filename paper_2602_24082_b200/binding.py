@@ -23,7 +23,7 @@ _lib: Optional[ctypes.CDLL] = None
 EXPORTS = ["pp_plan_workspace_bytes", "pp_build_plan", "pp_plan_status", "pp_destroy_plan",
            "pp_plan_max_tiles", "pp_plan_read", "pp_attn_fwd", "pp_attn_bwd",
            "pp_last_launch_count", "pp_error_string", "pp_step_host_arena_bytes", "pp_step_host_runs",
-           "pp_attn_step_host", "pp_profile_enable", "pp_profile_read",
+           "pp_attn_step_host", "pp_profile_enable", "pp_profile_read", "pp_profile_read_all",
            "pp_attn_bwd_noalloc", "pp_attn_bwd_noalloc_max_bytes", "pp_plan_read_bwd_units",
            "pp_plan_read_bwd_tiles", "pp_attn_bwd_deterministic",
            "pp_position_ids", "pp_rope_qk", "pp_preference_loss",
@@ -89,6 +89,7 @@ def lib() -> ctypes.CDLL:
         L.pp_preference_loss.argtypes = [vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp]
         L.pp_profile_enable.argtypes = [ctypes.c_int]
         L.pp_profile_read.argtypes = [vp, vp]
+        L.pp_profile_read_all.argtypes = [vp, vp, ctypes.c_int32, vp, vp]
         _lib = L
     return _lib
 
@@ -414,6 +415,17 @@ def pp_profile_read() -> Tuple[Optional[float], float]:
     _check(lib().pp_profile_read(ctypes.byref(a) if _profile_fwd else None, ctypes.byref(b)),
            "pp_profile_read")
     return (a.value if _profile_fwd else None), b.value
+
+
+def pp_profile_read_all(capacity: int = 64) -> Tuple[list, list]:
+    """(forward kernel ms, backward main kernel ms) of the most recent calls since the last
+    pp_profile_enable, oldest first (at most 64 each); sync the stream first."""
+    a = (ctypes.c_float * capacity)()
+    b = (ctypes.c_float * capacity)()
+    na, nb = ctypes.c_int32(0), ctypes.c_int32(0)
+    _check(lib().pp_profile_read_all(a if _profile_fwd else None, b, capacity,
+                                     ctypes.byref(na), ctypes.byref(nb)), "pp_profile_read_all")
+    return ([a[i] for i in range(na.value)] if _profile_fwd else []), [b[i] for i in range(nb.value)]
 
 
 def pp_last_launch_count() -> int:

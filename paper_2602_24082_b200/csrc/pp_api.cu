@@ -665,6 +665,16 @@ int pp_profile_read(float* fwd_kernel_ms, float* bwd_main_kernel_ms) {
   return pp::profile_read(fwd_kernel_ms, bwd_main_kernel_ms) ? PP_OK : PP_ERR_CUDA;
 }
 
+int pp_profile_read_all(float* fwd_kernel_ms, float* bwd_main_kernel_ms, int32_t capacity,
+                        int32_t* num_fwd, int32_t* num_bwd) {
+  if (capacity < 0) return PP_ERR_INVALID_ARG;
+  int nf = 0, nb = 0;
+  const bool ok = pp::profile_read_all(fwd_kernel_ms, bwd_main_kernel_ms, capacity, &nf, &nb);
+  if (num_fwd) *num_fwd = nf;
+  if (num_bwd) *num_bwd = nb;
+  return ok ? PP_OK : PP_ERR_CUDA;
+}
+
 int pp_build_rows_workspace_bytes(int32_t num_groups, size_t* bytes) {
   if (num_groups < 1 || !bytes) return PP_ERR_INVALID_ARG;
   *bytes = pp::rows_workspace_bytes(num_groups);

@@ -894,11 +894,12 @@ cudaError_t launch_bwd_t(const pp_plan* plan, const void* o, const float* lse, c
   const long long units = (long long)plan->max_tiles * pb.num_kv_heads;
   dim3 grid(unsigned(std::min<long long>(units, num_sms)));
   ProfileEvents& ev = profile_events();
-  if (ev.on) profile_record(ev.bwd0, stream);
+  const int slot = int(ev.bwd_count % kProfileRing);
+  if (ev.on) profile_record(ev.bwd0[slot], stream);
   kern<<<grid, kBwdThreads, BwdSmem<D>::kTotal, stream>>>(tq, tk, tv, tdo, tdq, prm);
   if (ev.on) {
-    profile_record(ev.bwd1, stream);
-    ev.bwd_valid = true;
+    profile_record(ev.bwd1[slot], stream);
+    ++ev.bwd_count;
   }
   const size_t n4 = T * Hq * DV / 4;
   unsigned fb = unsigned(std::min<size_t>((n4 + 255) / 256, size_t(num_sms) * 16));

@@ -700,11 +700,12 @@ cudaError_t launch_fwd_t(const pp_plan* plan, const CUtensorMap& tq, const CUten
   const long long units = (long long)plan->max_tiles * pb.num_kv_heads * ((r + 1) / 2);
   dim3 grid(unsigned(std::min<long long>(units, num_sms)));
   ProfileEvents& ev = profile_events();
-  if (ev.on && ev.fwd_on) profile_record(ev.fwd0, stream);
+  const int slot = int(ev.fwd_count % kProfileRing);
+  if (ev.on && ev.fwd_on) profile_record(ev.fwd0[slot], stream);
   kern<<<grid, kFwdThreads, FwdSmem<D>::kTotal, stream>>>(tq, tk, tv, prm);
   if (ev.on && ev.fwd_on) {
-    profile_record(ev.fwd1, stream);
-    ev.fwd_valid = true;
+    profile_record(ev.fwd1[slot], stream);
+    ++ev.fwd_count;
   }
   return cudaGetLastError();
 }

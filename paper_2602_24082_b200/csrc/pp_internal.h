@@ -197,11 +197,15 @@ inline bool device_is_sm100() {
 }
 
 // Optional event pairs around the forward kernel and the backward main kernel.
+// A ring of pairs per kernel, so that a benchmark can time many steps and read the durations
+// afterwards instead of synchronising after every step.
+constexpr int kProfileRing = 64;
 struct ProfileEvents {
   bool on = false;
   bool fwd_on = false;  // forward events wanted too (mode 1); mode 2 times the backward only
-  cudaEvent_t fwd0 = nullptr, fwd1 = nullptr, bwd0 = nullptr, bwd1 = nullptr;
-  bool fwd_valid = false, bwd_valid = false;
+  cudaEvent_t fwd0[kProfileRing] = {}, fwd1[kProfileRing] = {}, bwd0[kProfileRing] = {},
+              bwd1[kProfileRing] = {};
+  long long fwd_count = 0, bwd_count = 0;   // launches recorded since the events were enabled
 };
 ProfileEvents& profile_events();
 // Records a profiling event.  On a capturing stream the record becomes a node of the graph
@@ -215,6 +219,7 @@ inline void profile_record(cudaEvent_t ev, cudaStream_t stream) {
 }
 bool profile_enable(int mode);
 bool profile_read(float* fwd_ms, float* bwd_ms);
+bool profile_read_all(float* fwd_ms, float* bwd_ms, int capacity, int* n_fwd, int* n_bwd);
 
 // launchers (defined in the .cu files); all return a cudaError_t
 cudaError_t launch_plan(const pp_plan* plan, cudaStream_t stream, int* launches);

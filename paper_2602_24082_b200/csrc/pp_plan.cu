@@ -499,31 +499,61 @@ ProfileEvents& profile_events() {
 bool profile_enable(int mode) {
   ProfileEvents& ev = profile_events();
   const bool on = mode != 0;
-  if (on && ev.on) {  // already on: only the choice of kernels can change
+  if (on && ev.on) {  // already on: the choice of kernels can change, and the counts restart
     ev.fwd_on = mode == 1;
+    ev.fwd_count = ev.bwd_count = 0;
     return true;
   }
   if (on == ev.on) return true;
   if (on) {
-    bool ok = cudaEventCreate(&ev.fwd0) == cudaSuccess && cudaEventCreate(&ev.fwd1) == cudaSuccess &&
-              cudaEventCreate(&ev.bwd0) == cudaSuccess && cudaEventCreate(&ev.bwd1) == cudaSuccess;
+    bool ok = true;
+    for (int i = 0; i < kProfileRing && ok; ++i)
+      ok = cudaEventCreate(&ev.fwd0[i]) == cudaSuccess && cudaEventCreate(&ev.fwd1[i]) == cudaSuccess &&
+           cudaEventCreate(&ev.bwd0[i]) == cudaSuccess && cudaEventCreate(&ev.bwd1[i]) == cudaSuccess;
     ev.on = ok;
     ev.fwd_on = mode == 1;
-    ev.fwd_valid = ev.bwd_valid = false;
+    ev.fwd_count = ev.bwd_count = 0;
     return ok;
   }
-  cudaEventDestroy(ev.fwd0); cudaEventDestroy(ev.fwd1);
-  cudaEventDestroy(ev.bwd0); cudaEventDestroy(ev.bwd1);
+  for (int i = 0; i < kProfileRing; ++i) {
+    cudaEventDestroy(ev.fwd0[i]); cudaEventDestroy(ev.fwd1[i]);
+    cudaEventDestroy(ev.bwd0[i]); cudaEventDestroy(ev.bwd1[i]);
+  }
   ev = ProfileEvents();
   return true;
+}
+
+// Durations of the most recent launches, oldest first (at most kProfileRing are kept).
+bool profile_read_all(float* fwd_ms, float* bwd_ms, int capacity, int* n_fwd, int* n_bwd) {
+  ProfileEvents& ev = profile_events();
+  if (!ev.on || capacity < 0) return false;
+  bool ok = true;
+  auto dump = [&](float* out, int* n_out, long long count, cudaEvent_t* e0, cudaEvent_t* e1) {
+    const int n = int(std::min<long long>(std::min<long long>(count, kProfileRing), capacity));
+    if (n_out) *n_out = n;
+    if (!out) return;
+    for (int i = 0; i < n; ++i) {
+      const long long idx = count - n + i;
+      ok = ok && cudaEventElapsedTime(&out[i], e0[idx % kProfileRing], e1[idx % kProfileRing]) == cudaSuccess;
+    }
+  };
+  dump(fwd_ms, n_fwd, ev.fwd_count, ev.fwd0, ev.fwd1);
+  dump(bwd_ms, n_bwd, ev.bwd_count, ev.bwd0, ev.bwd1);
+  return ok;
 }
 
 bool profile_read(float* fwd_ms, float* bwd_ms) {
   ProfileEvents& ev = profile_events();
   if (!ev.on) return false;
   bool ok = true;
-  if (fwd_ms) ok = ok && ev.fwd_valid && cudaEventElapsedTime(fwd_ms, ev.fwd0, ev.fwd1) == cudaSuccess;
-  if (bwd_ms) ok = ok && ev.bwd_valid && cudaEventElapsedTime(bwd_ms, ev.bwd0, ev.bwd1) == cudaSuccess;
+  if (fwd_ms) {
+    const long long i = (ev.fwd_count - 1) % kProfileRing;
+    ok = ok && ev.fwd_count > 0 && cudaEventElapsedTime(fwd_ms, ev.fwd0[i], ev.fwd1[i]) == cudaSuccess;
+  }
+  if (bwd_ms) {
+    const long long i = (ev.bwd_count - 1) % kProfileRing;
+    ok = ok && ev.bwd_count > 0 && cudaEventElapsedTime(bwd_ms, ev.bwd0[i], ev.bwd1[i]) == cudaSuccess;
+  }
   return ok;
 }
 

@@ -278,3 +278,34 @@ def test_this_device_passes_the_compute_capability_check():
     assert torch.cuda.get_device_capability(0)[0] == 10
     plan = B.plan_for(W.config0())
     assert plan.status() == (0, 0)
+
+
+@pytest.mark.gpu
+def test_profile_event_ring():
+    """Kernel event timing over several calls without a synchronisation in between: the ring
+    returns one duration per call, oldest first, and restarts when profiling is re-enabled."""
+    from paper_2602_24082_b200 import binding as B
+    w = W.Workload("ring", [[(300, (140, 77))], [(64, (200, 1))]], 4, 2, 128, seed=3)
+    q, k, v, do = (x.cuda() for x in w.tensors())
+    plan = B.plan_for(w)
+    B.pp_profile_enable(True)
+    try:
+        for _ in range(5):
+            o, lse = B.pp_attn_fwd(plan, q, k, v, w.softmax_scale)
+            B.pp_attn_bwd(plan, q, k, v, o, lse, do, w.softmax_scale)
+        torch.cuda.synchronize()
+        f, b = B.pp_profile_read_all(64)
+        assert len(f) == 5 and len(b) == 5 and all(x > 0 for x in f + b)
+        last_f, last_b = B.pp_profile_read()
+        assert last_f == f[-1] and last_b == b[-1]
+        f2, b2 = B.pp_profile_read_all(3)
+        assert f2 == f[-3:] and b2 == b[-3:]
+        B.pp_profile_enable(True, backward_only=True)
+        o, lse = B.pp_attn_fwd(plan, q, k, v, w.softmax_scale)
+        B.pp_attn_bwd(plan, q, k, v, o, lse, do, w.softmax_scale)
+        torch.cuda.synchronize()
+        f3, b3 = B.pp_profile_read_all(64)
+        assert f3 == [] and len(b3) == 1
+    finally:
+        B.pp_profile_enable(False)
+    assert plan.status() == (0, 0)
